@@ -1,0 +1,169 @@
+/*
+ * rlhf_ppo.h -- C ABI of the token-level PPO math for RLHF on NVIDIA B200 (sm_100a).
+ *
+ * The PPO stage of RLHF (paper, Section 2.1 "RLHF Training") runs four models: the actor, the
+ * frozen reference that keeps the reward from diverging, the reward model that scores a whole
+ * sequence, and the critic that estimates returns.  The actor generates responses; inference
+ * passes of the four models turn them into experience; then the actor is trained to raise reward
+ * while limiting its deviation from the old policy, and the critic is trained on the returns.
+ * This library is the math between the models' outputs and their backward passes:
+ *
+ *   rlhf_gather_logprobs    log-prob of each generated token from a logits tensor (actor, reference)
+ *   rlhf_kl_reward          per-token reward: KL penalty against the reference + sequence score
+ *   rlhf_gae                advantages and returns from rewards and critic values
+ *   rlhf_ppo_loss_fwd_bwd   clipped policy and value loss, gradient w.r.t. the logits and values
+ *
+ * The paper gives these quantities in prose only; the formulas are the standard definitions and
+ * are written out beside each function.
+ *
+ * Conventions
+ *  - B sequences, T response positions, V vocabulary entries.  lengths[b] in [0,T] is the number
+ *    of valid response tokens of sequence b; positions t >= lengths[b] are padding.  Padded
+ *    positions are ignored on input and every output is written as 0 there.
+ *    N = sum_b lengths[b].
+ *  - Every pointer is a DEVICE pointer owned by the caller unless it says "host".  The library
+ *    allocates nothing, frees nothing and keeps no state between calls.  Calls are asynchronous
+ *    on `stream` (a cudaStream_t passed as void*, NULL = the default stream) and never
+ *    synchronise it (rlhf_poll_status excepted).
+ *  - [B,T] arrays are fp32 (ids int64, lengths int32), row-major, T contiguous.
+ *  - Logits are bf16, addressed as base[b*stride_b + t*stride_t + v], strides in ELEMENTS,
+ *    stride_t >= V.  For a full-sequence tensor [B,P+T,V] whose row P-1+t predicts response
+ *    token t, pass base + (P-1)*V, stride_b = (P+T)*V, stride_t = V, and ids = input_ids + P with
+ *    ids_stride_b = P+T.  Rows whose start address and byte length are multiples of 16 take the
+ *    fast path; any other layout is handled by a slower kernel, not rejected.
+ *  - A logit of -inf is a deleted vocabulary entry (probability 0, gradient 0).  It must not be
+ *    the generated token's logit and a row must keep at least one finite logit; finite logits
+ *    must satisfy |z| <= 1e38.  Violations produce NaN/inf in that row's outputs, never a fault.
+ *  - Return value: an rlhf_status_t.  Errors the host can see (null pointers, sizes, strides,
+ *    scalars out of range, workspace too small) are returned at once and nothing is launched.
+ *    Errors only the device can see (an id outside [0,V), a length outside [0,T], a bounded wait
+ *    that ran out) never fault: the offending token is treated as padding (length clamped), the
+ *    code is OR-ed into the first word of the workspace, and rlhf_poll_status reports it.
+ *  - Arithmetic: fp32 throughout (exp/log of the softmax in base 2 with the hardware ex2); bf16
+ *    outputs are rounded to nearest even.  Results do not depend on the order in which rows are
+ *    scheduled: the loss is reduced in a fixed order, without floating-point atomics.
+ */
+#ifndef RLHF_PPO_H_
+#define RLHF_PPO_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RLHF_OK = 0,
+    RLHF_ERR_NULL = 1,          /* a required pointer is NULL */
+    RLHF_ERR_SHAPE = 2,         /* B, T or V <= 0, or B*T too large */
+    RLHF_ERR_ALIGN = 3,         /* a [B,T] array or the workspace is not aligned to its element / 256 B */
+    RLHF_ERR_STRIDE = 4,        /* stride_t < V, negative stride, rows of different sequences overlap */
+    RLHF_ERR_WORKSPACE = 5,     /* workspace smaller than rlhf_workspace_bytes(B,T) */
+    RLHF_ERR_SCALAR = 6,        /* non-finite or out-of-range scalar argument */
+    RLHF_ERR_CUDA = 7,          /* a CUDA runtime call or launch failed; see rlhf_last_cuda_error */
+    /* device-detected, sticky in the workspace, bit flags (may be OR-ed together) */
+    RLHF_ERR_ID_RANGE = 16,     /* a generated-token id outside [0,V) at a valid position */
+    RLHF_ERR_LENGTH_RANGE = 32, /* a length outside [0,T] (clamped) */
+    RLHF_ERR_TIMEOUT = 64       /* an internal bounded wait ran out; outputs of this call are invalid */
+} rlhf_status_t;
+
+/* Human-readable name of a status (static storage; flags are joined with '|'). Host, never NULL. */
+const char* rlhf_status_string(int status);
+
+/* Text of the last CUDA runtime error this library saw on the calling thread ("" if none). */
+const char* rlhf_last_cuda_error(void);
+
+/* Bytes of scratch that rlhf_gather_logprobs and rlhf_ppo_loss_fwd_bwd need for a batch of B x T
+ * tokens: O(B*T), never O(B*T*V) -- at most 16*B*T + 65536.  0 if B or T is not positive.
+ * The workspace must be 256-byte aligned and must have been cleared once with rlhf_workspace_init
+ * before its first use; it can then be reused by any number of calls on the same stream. */
+size_t rlhf_workspace_bytes(int B, int T);
+
+/* Zero the workspace (asynchronously, on `stream`). Needed once after allocation. */
+int rlhf_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronise `stream`, return the device-detected status flags accumulated in the workspace since
+ * the last poll (RLHF_OK if none) and clear them. */
+int rlhf_poll_status(void* workspace, void* stream);
+
+/*
+ * Step 1 -- log-probability of the generated tokens (Section 2.1: the actor and reference
+ * inferences that produce the experience).  For t < lengths[b], with z = logits[b,t,:], y = ids[b,t]:
+ *     out_logprobs[b,t] = z_y - log sum_v exp(z_v)
+ * and 0 for t >= lengths[b].  One streaming read of each valid row; padded rows are not read.
+ *   logits        bf16 [B,T,V] through (stride_b, stride_t)             read
+ *   ids           int64, ids[b*ids_stride_b + t]                        read
+ *   lengths       int32 [B]                                             read
+ *   out_logprobs  fp32 [B,T]                                            written (all B*T entries)
+ *   workspace     >= rlhf_workspace_bytes(B,T), 256-B aligned, initialised
+ */
+int rlhf_gather_logprobs(const void* logits, long long stride_b, long long stride_t,
+                         const long long* ids, long long ids_stride_b, const int* lengths,
+                         int B, int T, int V, float* out_logprobs,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Step 2 -- per-token reward (Section 2.1: the reference model prevents reward divergence, the
+ * reward model gives the sequence-level score).  For t < lengths[b]:
+ *     out_rewards[b,t] = -beta_kl * (lp_old[b,t] - lp_ref[b,t])
+ *                        + [t == lengths[b]-1] * clamp(score[b], -reward_clip, +reward_clip)
+ * and 0 for t >= lengths[b].  lp_old are the actor's log-probs when the experience was made.
+ *   lp_old, lp_ref  fp32 [B,T]; score fp32 [B]; lengths int32 [B]      read
+ *   out_rewards     fp32 [B,T]                                         written; may alias lp_old or lp_ref
+ *   beta_kl >= 0, reward_clip >= 0 (use a huge value for "no clip"); both finite.
+ */
+int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score, const int* lengths,
+                   int B, int T, float beta_kl, float reward_clip, float* out_rewards, void* stream);
+
+/*
+ * Step 3 -- generalised advantage estimation (Section 2.1: the critic estimates returns).
+ * Backwards from the last valid token, with V_len = A_len = 0:
+ *     delta_t = r_t + gamma * V_{t+1} - V_t
+ *     A_t     = delta_t + gamma * lambda * A_{t+1}
+ *     G_t     = A_t + V_t
+ * out_adv = A, out_returns = G, both 0 for t >= lengths[b].
+ *   rewards, values_old  fp32 [B,T]; lengths int32 [B]                  read
+ *   out_adv, out_returns fp32 [B,T]                                     written; must not alias the inputs
+ *   gamma, lambda in [0,1].
+ */
+int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, int B, int T,
+             float gamma, float lambda, float* out_adv, float* out_returns, void* stream);
+
+/*
+ * Step 4 -- clipped PPO losses and their gradients (Section 2.1: the actor is trained to maximise
+ * reward while limiting policy deviation, the critic is trained on the returns).  For each valid
+ * token, with lp_new = z_y - lse(z) from the current logits (as step 1), rho = exp(lp_new - lp_old):
+ *     l_pg = max(-A*rho, -A*clamp(rho, 1-clip_eps, 1+clip_eps))
+ *     g    = grad_scale * (-A*rho) / N   if -A*rho >= -A*clamp(rho, ...)   else 0
+ *     out_dlogits[b,t,v] = bf16( g * ([v == y] - exp(z_v - lse)) )
+ *     vc   = values_old + clamp(values_new - values_old, -value_clip, +value_clip)
+ *     l_vf = 1/2 * max((values_new - G)^2, (vc - G)^2)
+ *     out_dvalues[b,t] = grad_scale * (values_new - G) / N   if (values_new-G)^2 >= (vc-G)^2   else 0
+ *     *out_loss_pg = (1/N) sum l_pg        *out_loss_vf = (1/N) sum l_vf
+ * Padded rows of out_dlogits are written as zeros, padded out_dvalues / out_lp_new as 0.  If N = 0
+ * both losses and all gradients are 0.  Each valid row is read once from DRAM and written once.
+ *   logits                       bf16 via (stride_b, stride_t)          read
+ *   ids, lengths                 as step 1                              read
+ *   lp_old, adv, values_new, values_old, returns   fp32 [B,T]           read
+ *   out_loss_pg, out_loss_vf     fp32 scalars (device)                  written
+ *   out_dlogits                  bf16 via (dl_stride_b, dl_stride_t)    written (all B*T rows); may be the
+ *                                logits buffer itself with the same strides (in place), must not
+ *                                otherwise overlap it
+ *   out_dvalues                  fp32 [B,T]                             written
+ *   out_lp_new                   fp32 [B,T] or NULL                     written if given
+ *   clip_eps in (0,1), value_clip >= 0, grad_scale finite.
+ */
+int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stride_t,
+                          const long long* ids, long long ids_stride_b, const int* lengths,
+                          const float* lp_old, const float* adv, const float* values_new,
+                          const float* values_old, const float* returns,
+                          int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
+                          float* out_loss_pg, float* out_loss_vf,
+                          void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                          float* out_dvalues, float* out_lp_new,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RLHF_PPO_H_ */

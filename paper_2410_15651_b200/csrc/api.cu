@@ -1,0 +1,287 @@
+// C ABI of the token-level PPO library: argument checks and kernel launches.
+// Declarations and the meaning of every argument are in include/rlhf_ppo.h.
+#include "../../include/rlhf_ppo.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "kernels_generic.cuh"
+#include "kernels_small.cuh"
+
+namespace {
+
+using namespace rlhf;
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what)
+{
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    return RLHF_ERR_CUDA;
+}
+
+#define RLHF_CUDA(call)                                   \
+    do {                                                  \
+        cudaError_t e_ = (call);                          \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+// Workspace layout (bytes): [0,4) status flags, [4,8) finalisation ticket, [256, 256+4096) block
+// partials of the finalisation (256 blocks x 2 doubles), [kRowLossOffset, +4*B*T) per-token policy
+// loss terms.
+constexpr size_t kPartialsOffset = 256;
+constexpr size_t kRowLossOffset = 8192;
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_shape(int B, int T, int V)
+{
+    if (B <= 0 || T <= 0 || V <= 0) return RLHF_ERR_SHAPE;
+    if ((long long)B * (long long)T > (1ll << 30)) return RLHF_ERR_SHAPE;
+    return RLHF_OK;
+}
+
+int check_workspace(const void* ws, size_t bytes, int B, int T)
+{
+    if (!ws) return RLHF_ERR_NULL;
+    if (!aligned(ws, 256)) return RLHF_ERR_ALIGN;
+    if (bytes < rlhf_workspace_bytes(B, T)) return RLHF_ERR_WORKSPACE;
+    return RLHF_OK;
+}
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int max_smem_optin = 0;
+};
+
+// Queried per call: the library keeps no state, and the two attributes are cheap to read.
+int device_info(DeviceInfo& d)
+{
+    int dev = 0;
+    RLHF_CUDA(cudaGetDevice(&dev));
+    RLHF_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    RLHF_CUDA(cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    return RLHF_OK;
+}
+
+int launch_check(const char* what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, what);
+    return RLHF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rlhf_status_string(int status)
+{
+    switch (status) {
+        case RLHF_OK: return "RLHF_OK";
+        case RLHF_ERR_NULL: return "RLHF_ERR_NULL";
+        case RLHF_ERR_SHAPE: return "RLHF_ERR_SHAPE";
+        case RLHF_ERR_ALIGN: return "RLHF_ERR_ALIGN";
+        case RLHF_ERR_STRIDE: return "RLHF_ERR_STRIDE";
+        case RLHF_ERR_WORKSPACE: return "RLHF_ERR_WORKSPACE";
+        case RLHF_ERR_SCALAR: return "RLHF_ERR_SCALAR";
+        case RLHF_ERR_CUDA: return "RLHF_ERR_CUDA";
+        default: break;
+    }
+    if (status > 0 && (status & ~(RLHF_ERR_ID_RANGE | RLHF_ERR_LENGTH_RANGE | RLHF_ERR_TIMEOUT)) == 0) {
+        static const char* const names[8] = {
+            "RLHF_OK",
+            "RLHF_ERR_ID_RANGE",
+            "RLHF_ERR_LENGTH_RANGE",
+            "RLHF_ERR_ID_RANGE|RLHF_ERR_LENGTH_RANGE",
+            "RLHF_ERR_TIMEOUT",
+            "RLHF_ERR_ID_RANGE|RLHF_ERR_TIMEOUT",
+            "RLHF_ERR_LENGTH_RANGE|RLHF_ERR_TIMEOUT",
+            "RLHF_ERR_ID_RANGE|RLHF_ERR_LENGTH_RANGE|RLHF_ERR_TIMEOUT",
+        };
+        return names[(status >> 4) & 7];
+    }
+    return "RLHF_ERR_UNKNOWN";
+}
+
+const char* rlhf_last_cuda_error(void) { return g_cuda_error; }
+
+size_t rlhf_workspace_bytes(int B, int T)
+{
+    if (B <= 0 || T <= 0) return 0;
+    size_t n = kRowLossOffset + 4 * (size_t)B * (size_t)T;
+    return (n + 255) & ~(size_t)255;
+}
+
+int rlhf_workspace_init(void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!workspace) return RLHF_ERR_NULL;
+    if (!aligned(workspace, 256)) return RLHF_ERR_ALIGN;
+    if (workspace_bytes < kRowLossOffset) return RLHF_ERR_WORKSPACE;
+    RLHF_CUDA(cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream));
+    return RLHF_OK;
+}
+
+int rlhf_poll_status(void* workspace, void* stream)
+{
+    if (!workspace) return RLHF_ERR_NULL;
+    unsigned flags = 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    RLHF_CUDA(cudaMemcpyAsync(&flags, workspace, sizeof flags, cudaMemcpyDeviceToHost, s));
+    RLHF_CUDA(cudaStreamSynchronize(s));
+    if (flags != 0) {
+        RLHF_CUDA(cudaMemsetAsync(workspace, 0, sizeof flags, s));
+        RLHF_CUDA(cudaStreamSynchronize(s));
+    }
+    return (int)flags;
+}
+
+int rlhf_gather_logprobs(const void* logits, long long stride_b, long long stride_t,
+                         const long long* ids, long long ids_stride_b, const int* lengths,
+                         int B, int T, int V, float* out_logprobs,
+                         void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!logits || !ids || !lengths || !out_logprobs) return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, V)) return e;
+    if (stride_b < 0 || stride_t < 0 || ids_stride_b < 0) return RLHF_ERR_STRIDE;
+    if (T > 1 && stride_t < V) return RLHF_ERR_STRIDE;
+    if (!aligned(logits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) || !aligned(out_logprobs, 4))
+        return RLHF_ERR_ALIGN;
+    if (int e = check_workspace(workspace, workspace_bytes, B, T)) return e;
+    DeviceInfo dev;
+    if (int e = device_info(dev)) return e;
+
+    RowArgs a{};
+    a.logits = (const uint16_t*)logits;
+    a.stride_b = stride_b;
+    a.stride_t = stride_t;
+    a.ids = ids;
+    a.ids_stride_b = ids_stride_b;
+    a.lengths = lengths;
+    a.B = B; a.T = T; a.V = V;
+    a.status = (unsigned*)workspace;
+    a.out_lp = out_logprobs;
+
+    long long rows = (long long)B * T;
+    int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
+    row_generic_kernel<false><<<grid, kGenericThreads, 0, (cudaStream_t)stream>>>(a);
+    return launch_check("row_generic_kernel<logprob>");
+}
+
+int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score, const int* lengths,
+                   int B, int T, float beta_kl, float reward_clip, float* out_rewards, void* stream)
+{
+    if (!lp_old || !lp_ref || !score || !lengths || !out_rewards) return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, 1)) return e;
+    if (!std::isfinite(beta_kl) || beta_kl < 0.f || !std::isfinite(reward_clip) || reward_clip < 0.f)
+        return RLHF_ERR_SCALAR;
+    if (!aligned(lp_old, 4) || !aligned(lp_ref, 4) || !aligned(score, 4) || !aligned(lengths, 4) ||
+        !aligned(out_rewards, 4))
+        return RLHF_ERR_ALIGN;
+    long long total = (long long)B * T;
+    int grid = (int)std::min<long long>((total + 255) / 256, 1184);
+    kl_reward_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(lp_old, lp_ref, score, lengths, B, T,
+                                                           beta_kl, reward_clip, out_rewards);
+    return launch_check("kl_reward_kernel");
+}
+
+int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, int B, int T,
+             float gamma, float lambda, float* out_adv, float* out_returns, void* stream)
+{
+    if (!rewards || !values_old || !lengths || !out_adv || !out_returns) return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, 1)) return e;
+    if (!(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f)) return RLHF_ERR_SCALAR;
+    if (!aligned(rewards, 4) || !aligned(values_old, 4) || !aligned(lengths, 4) || !aligned(out_adv, 4) ||
+        !aligned(out_returns, 4))
+        return RLHF_ERR_ALIGN;
+    if (out_adv == rewards || out_adv == values_old || out_returns == rewards ||
+        out_returns == values_old || out_adv == out_returns)
+        return RLHF_ERR_STRIDE;
+    int grid = (B + kGaeWarpsPerBlock - 1) / kGaeWarpsPerBlock;
+    gae_kernel<<<grid, kGaeWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(rewards, values_old, lengths, B, T,
+                                                                       gamma, lambda, out_adv, out_returns);
+    return launch_check("gae_kernel");
+}
+
+int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stride_t,
+                          const long long* ids, long long ids_stride_b, const int* lengths,
+                          const float* lp_old, const float* adv, const float* values_new,
+                          const float* values_old, const float* returns,
+                          int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
+                          float* out_loss_pg, float* out_loss_vf,
+                          void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                          float* out_dvalues, float* out_lp_new,
+                          void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!logits || !ids || !lengths || !lp_old || !adv || !values_new || !values_old || !returns ||
+        !out_loss_pg || !out_loss_vf || !out_dlogits || !out_dvalues)
+        return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, V)) return e;
+    if (stride_b < 0 || stride_t < 0 || ids_stride_b < 0 || dl_stride_b < 0 || dl_stride_t < 0)
+        return RLHF_ERR_STRIDE;
+    if (T > 1 && (stride_t < V || dl_stride_t < V)) return RLHF_ERR_STRIDE;
+    if (B > 1 && dl_stride_b < (long long)(T - 1) * dl_stride_t + V) return RLHF_ERR_STRIDE;
+    if (out_dlogits == logits && (dl_stride_b != stride_b || dl_stride_t != stride_t)) return RLHF_ERR_STRIDE;
+    if (!(clip_eps > 0.f && clip_eps < 1.f) || !std::isfinite(value_clip) || value_clip < 0.f ||
+        !std::isfinite(grad_scale))
+        return RLHF_ERR_SCALAR;
+    if (!aligned(logits, 2) || !aligned(out_dlogits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) ||
+        !aligned(lp_old, 4) || !aligned(adv, 4) || !aligned(values_new, 4) || !aligned(values_old, 4) ||
+        !aligned(returns, 4) || !aligned(out_loss_pg, 4) || !aligned(out_loss_vf, 4) ||
+        !aligned(out_dvalues, 4) || (out_lp_new && !aligned(out_lp_new, 4)))
+        return RLHF_ERR_ALIGN;
+    if (int e = check_workspace(workspace, workspace_bytes, B, T)) return e;
+    DeviceInfo dev;
+    if (int e = device_info(dev)) return e;
+
+    char* ws = (char*)workspace;
+    RowArgs a{};
+    a.logits = (const uint16_t*)logits;
+    a.stride_b = stride_b;
+    a.stride_t = stride_t;
+    a.ids = ids;
+    a.ids_stride_b = ids_stride_b;
+    a.lengths = lengths;
+    a.B = B; a.T = T; a.V = V;
+    a.status = (unsigned*)ws;
+    a.lp_old = lp_old;
+    a.adv = adv;
+    a.clip_eps = clip_eps;
+    a.grad_scale = grad_scale;
+    a.dlogits = (uint16_t*)out_dlogits;
+    a.dl_stride_b = dl_stride_b;
+    a.dl_stride_t = dl_stride_t;
+    a.row_loss = (float*)(ws + kRowLossOffset);
+    a.out_lp_new = out_lp_new;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    long long rows = (long long)B * T;
+    int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
+    row_generic_kernel<true><<<grid, kGenericThreads, 0, s>>>(a);
+    if (int e = launch_check("row_generic_kernel<loss>")) return e;
+
+    FinalArgs f{};
+    f.lengths = lengths;
+    f.B = B; f.T = T;
+    f.values_new = values_new;
+    f.values_old = values_old;
+    f.returns = returns;
+    f.row_loss = a.row_loss;
+    f.value_clip = value_clip;
+    f.grad_scale = grad_scale;
+    f.out_dvalues = out_dvalues;
+    f.out_lp_new = out_lp_new;
+    f.out_loss_pg = out_loss_pg;
+    f.out_loss_vf = out_loss_vf;
+    f.status = (unsigned*)ws;
+    f.ticket = (unsigned*)(ws + 4);
+    f.partials = (double*)(ws + kPartialsOffset);
+    int fgrid = (int)std::min<long long>((rows + 1023) / 1024, kFinalMaxBlocks);
+    ppo_finalize_kernel<<<fgrid, kFinalThreads, 0, s>>>(f);
+    return launch_check("ppo_finalize_kernel");
+}
+
+}  // extern "C"

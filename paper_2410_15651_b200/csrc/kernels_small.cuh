@@ -1,0 +1,173 @@
+// The O(B*T) kernels: per-token reward, GAE reverse scan, and the loss finalisation
+// (value loss, dvalues, deterministic reduction of both losses).
+#pragma once
+#include "common.cuh"
+
+namespace rlhf {
+
+// ---------------------------------------------------------------- step 2: per-token reward
+__global__ void __launch_bounds__(256) kl_reward_kernel(const float* __restrict__ lp_old,
+                                                        const float* __restrict__ lp_ref,
+                                                        const float* __restrict__ score,
+                                                        const int* __restrict__ lengths, int B, int T,
+                                                        float beta, float clip, float* out)
+{
+    const long long total = (long long)B * T;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        int b = (int)(i / T), t = (int)(i % T);
+        int len = clamp_len(__ldg(lengths + b), T);
+        float r = 0.f;
+        if (t < len) {
+            r = -beta * (lp_old[i] - lp_ref[i]);
+            if (t == len - 1) r += fminf(fmaxf(__ldg(score + b), -clip), clip);
+        }
+        out[i] = r;
+    }
+}
+
+// ---------------------------------------------------------------- step 3: GAE
+// One warp per sequence.  The recurrence A_t = delta_t + q A_{t+1} (q = gamma*lambda) is an affine
+// map of A_{t+1}; each lane composes the maps of its contiguous chunk of the valid range, a
+// 5-step shuffle suffix scan composes the chunks, and each lane then replays its chunk from the
+// now-known incoming value.  delta_t = r_t + gamma V_{t+1} - V_t with V_len = 0.
+constexpr int kGaeWarpsPerBlock = 4;
+
+__global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) gae_kernel(const float* __restrict__ rewards,
+                                                                     const float* __restrict__ values,
+                                                                     const int* __restrict__ lengths,
+                                                                     int B, int T, float gamma, float lambda,
+                                                                     float* __restrict__ adv,
+                                                                     float* __restrict__ ret)
+{
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kGaeWarpsPerBlock + (threadIdx.x >> 5);
+    if (b >= B) return;
+    const int n = clamp_len(__ldg(lengths + b), T);
+    const float* r = rewards + (long long)b * T;
+    const float* v = values + (long long)b * T;
+    float* a_out = adv + (long long)b * T;
+    float* g_out = ret + (long long)b * T;
+    const float q = gamma * lambda;
+
+    const int chunk = (n + 31) / 32;
+    const int lo = min(n, lane * chunk), hi = min(n, lo + chunk);
+
+    // chunk map: A_lo = P + c * A_hi
+    float P = 0.f, c = 1.f;
+    {
+        float v_next = hi < n ? v[hi] : 0.f;
+        for (int t = hi - 1; t >= lo; --t) {
+            float vt = v[t];
+            float delta = r[t] + gamma * v_next - vt;
+            P = fmaf(q, P, delta);
+            c *= q;
+            v_next = vt;
+        }
+    }
+    // suffix scan over lanes: (P,c) of lane l becomes the map of chunks l..31
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        float P2 = __shfl_down_sync(0xffffffffu, P, o);
+        float c2 = __shfl_down_sync(0xffffffffu, c, o);
+        if (lane + o < 32) { P = fmaf(c, P2, P); c *= c2; }
+    }
+    float a = __shfl_down_sync(0xffffffffu, P, 1);     // A at this lane's hi = A_lo of the next chunk
+    if (lane == 31) a = 0.f;
+    {
+        float v_next = hi < n ? v[hi] : 0.f;
+        for (int t = hi - 1; t >= lo; --t) {
+            float vt = v[t];
+            float delta = r[t] + gamma * v_next - vt;
+            a = fmaf(q, a, delta);
+            a_out[t] = a;
+            g_out[t] = a + vt;
+            v_next = vt;
+        }
+    }
+    for (int t = n + lane; t < T; t += 32) { a_out[t] = 0.f; g_out[t] = 0.f; }
+}
+
+// ---------------------------------------------------------------- step 4: finalisation
+// Value loss and dvalues per token, then both losses summed in a fixed order: each block reduces a
+// contiguous range of tokens with a fixed tree, the last block to finish (a ticket in the workspace)
+// adds the block partials in index order.  No floating-point atomics, so the result is bit-stable.
+constexpr int kFinalThreads = 256;
+constexpr int kFinalMaxBlocks = 256;
+
+struct FinalArgs {
+    const int* lengths;
+    int B, T;
+    const float* values_new;
+    const float* values_old;
+    const float* returns;
+    const float* row_loss;      // per-token policy loss terms written by the row kernel (valid tokens)
+    float value_clip, grad_scale;
+    float* out_dvalues;
+    float* out_lp_new;          // optional: zeroed at padded tokens here
+    float* out_loss_pg;
+    float* out_loss_vf;
+    unsigned* status;
+    unsigned* ticket;           // workspace word, zero between calls
+    double* partials;           // workspace: [kFinalMaxBlocks][2]
+};
+
+__global__ void __launch_bounds__(kFinalThreads) ppo_finalize_kernel(FinalArgs p)
+{
+    __shared__ long long s_cnt[33];
+    __shared__ double s_red[2][kFinalThreads / 32];
+    __shared__ bool s_last;
+    const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, nullptr);
+    const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
+
+    const long long total = (long long)p.B * p.T;
+    const long long per_block = (total + gridDim.x - 1) / gridDim.x;
+    const long long begin = per_block * blockIdx.x, end = min(total, begin + per_block);
+    double sum_pg = 0.0, sum_vf = 0.0;
+    for (long long i = begin + threadIdx.x; i < end; i += blockDim.x) {
+        int b = (int)(i / p.T), t = (int)(i % p.T);
+        float dv = 0.f;
+        if (t < clamp_len(__ldg(p.lengths + b), p.T)) {
+            float v = p.values_new[i], vo = p.values_old[i], G = p.returns[i];
+            float vc = vo + fminf(fmaxf(v - vo, -p.value_clip), p.value_clip);
+            float e1 = (v - G) * (v - G), e2 = (vc - G) * (vc - G);
+            if (e1 >= e2) { sum_vf += 0.5 * (double)e1; dv = (v - G) * scale_over_N; }
+            else sum_vf += 0.5 * (double)e2;
+            sum_pg += (double)p.row_loss[i];
+        } else if (p.out_lp_new) {
+            p.out_lp_new[i] = 0.f;
+        }
+        p.out_dvalues[i] = dv;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sum_pg += __shfl_xor_sync(0xffffffffu, sum_pg, o);
+        sum_vf += __shfl_xor_sync(0xffffffffu, sum_vf, o);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_red[0][warp] = sum_pg; s_red[1][warp] = sum_vf; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, c = 0.0;
+        for (int w = 0; w < kFinalThreads / 32; ++w) { a += s_red[0][w]; c += s_red[1][w]; }
+        p.partials[2 * blockIdx.x] = a;
+        p.partials[2 * blockIdx.x + 1] = c;
+        __threadfence();
+        unsigned prev = atomicAdd(p.ticket, 1u);
+        s_last = (prev == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (s_last && threadIdx.x == 0) {
+        __threadfence();
+        double a = 0.0, c = 0.0;
+        for (unsigned k = 0; k < gridDim.x; ++k) {
+            a += ((volatile double*)p.partials)[2 * k];
+            c += ((volatile double*)p.partials)[2 * k + 1];
+        }
+        *p.out_loss_pg = N > 0 ? (float)(a / (double)N) : 0.f;
+        *p.out_loss_vf = N > 0 ? (float)(c / (double)N) : 0.f;
+        *p.ticket = 0u;
+    }
+}
+
+}  // namespace rlhf

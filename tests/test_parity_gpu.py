@@ -1,0 +1,224 @@
+"""CUDA path against the CPU oracle, step by step, on the synthetic workloads.
+
+Each step of the CUDA library is given the same float32 inputs as the oracle (the oracle's own
+outputs of the step before, rounded to float32) and compared element by element.  The tiny case
+is compared in full; the larger ones in full for every O(B*T) output and on sampled rows for the
+bf16 logits gradient, plus properties that hold for every row.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2410_15651_b200 import binding, inputs
+
+from helpers import OracleRun, TOL_LP, check_dlogits_rows, close_rel, np32
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _t(a, dtype=torch.float32):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype, device=DEV)
+
+
+def run_steps(oracle, w, batch, run, logits, ref, ids, in_place=False, sample_rows=None, all_rows=False):
+    """Run every CUDA step on the oracle-fed inputs and compare.  Returns a dict of error ratios."""
+    B, T, V = logits.shape
+    lengths = batch["lengths"]
+    ws = binding.workspace(B, T, DEV)
+    report = {}
+
+    # step 1, actor and reference
+    lp_a = binding.gather_logprobs(logits, ids, lengths, ws)
+    lp_r = binding.gather_logprobs(ref, ids, lengths, ws)
+    for name, got, want in (("lp_actor", lp_a, run.lp_actor), ("lp_ref", lp_r, run.lp_ref)):
+        err = np.abs(np32(got).astype(np.float64) - want)
+        assert np.isfinite(np32(got)).all(), name
+        assert err.max(initial=0.0) <= TOL_LP, (name, err.max())
+        assert (np32(got)[~run.valid] == 0).all(), name
+        report[name] = err.max(initial=0.0) / TOL_LP
+
+    # step 2
+    r = binding.kl_reward(_t(run.lp_old_in), _t(run.lp_ref_in), _t(run.score_in), lengths,
+                          w.beta_kl, w.reward_clip)
+    ok, report["rewards"] = close_rel(np32(r), run.rewards)
+    assert ok, report
+    assert (np32(r)[~run.valid] == 0).all()
+
+    # step 3
+    adv, ret = binding.gae(_t(run.rewards_in), _t(run.values_old_in), lengths, w.gamma, w.lam)
+    ok, report["adv"] = close_rel(np32(adv), run.adv)
+    assert ok, report
+    ok, report["ret"] = close_rel(np32(ret), run.ret)
+    assert ok, report
+    assert (np32(adv)[~run.valid] == 0).all() and (np32(ret)[~run.valid] == 0).all()
+
+    # step 4
+    src = logits.clone() if in_place else logits
+    out = binding.PPOOutputs(src, in_place=in_place)
+    binding.ppo_loss_fwd_bwd(src, ids, lengths, _t(run.lp_old_in), _t(run.adv_in), _t(run.values_new_in),
+                             _t(run.values_old_in), _t(run.ret_in), w.clip_eps, w.value_clip,
+                             run.grad_scale, ws, out)
+    assert binding.poll_status(ws) == 0
+    loss = np32(out.loss).astype(np.float64)
+    ok, report["loss_pg"] = close_rel(loss[0], run.ppo.loss_pg)
+    assert ok, (loss, run.ppo.loss_pg, report)
+    ok, report["loss_vf"] = close_rel(loss[1], run.ppo.loss_vf)
+    assert ok, (loss, run.ppo.loss_vf, report)
+    lp_new = np32(out.lp_new).astype(np.float64)
+    assert np.abs(lp_new - run.lp_actor).max(initial=0.0) <= TOL_LP
+    assert (lp_new[~run.valid] == 0).all()
+    dv = np32(out.dvalues).astype(np.float64)
+    keep = ~run.vf_kink
+    ok, report["dvalues"] = close_rel(dv[keep], run.ppo.dvalues[keep])
+    assert ok, report
+    assert (dv[~run.valid] == 0).all()
+
+    rows = np.arange(B * T) if all_rows else np.asarray(sample_rows)
+    report["dlogits"], report["dlogits_rows"] = check_dlogits_rows(oracle, run, logits, ids, out.dlogits, rows)
+    return out, report
+
+
+def sample_rows(run, n, seed=0):
+    """A mix of valid rows, padded rows and zero-gradient rows."""
+    rng = np.random.default_rng(seed)
+    flat_valid = np.flatnonzero(run.valid.reshape(-1))
+    flat_pad = np.flatnonzero(~run.valid.reshape(-1))
+    zero_g = np.flatnonzero((run.ppo.g.reshape(-1) == 0) & run.valid.reshape(-1))
+    picks = [rng.choice(flat_valid, size=min(n, flat_valid.size), replace=False)]
+    if flat_pad.size:
+        picks.append(rng.choice(flat_pad, size=min(max(2, n // 8), flat_pad.size), replace=False))
+    if zero_g.size:
+        picks.append(zero_g[:4])
+    # first and last valid row, and the rows around each sequence end
+    picks.append(flat_valid[[0, -1]])
+    return np.unique(np.concatenate(picks))
+
+
+def dlogits_properties(run, out, ids, logits):
+    """Properties of the full dlogits tensor that need no oracle row: padded rows are zero, every
+    row sums to ~0 (within the bf16 rounding of its entries), the label entry carries the sign of g."""
+    B, T, V = logits.shape
+    d = out.dlogits
+    valid = torch.as_tensor(run.valid, device=d.device)
+    for b in range(B):
+        db = d[b].float()                                           # [T,V]
+        assert torch.isfinite(db).all()
+        pad = ~valid[b]
+        if pad.any():
+            assert (d[b][pad].view(torch.int16) == 0).all()         # exact +0
+        rs = db.double().sum(-1).abs()
+        lim = 0.5 * db.abs().double().sum(-1) * 2.0 ** -7 + 1e-5    # sum of half-ulps bound, with slack
+        assert (rs <= lim).all(), (b, float((rs / lim).max()))
+        g = torch.as_tensor(run.ppo.g[b], device=d.device)
+        dy = db.gather(1, ids[b][:, None])[:, 0].double()
+        # one_m_py can underflow to 0 for extremely peaked rows; otherwise the sign follows g
+        assert ((torch.sign(dy) == torch.sign(g)) | (dy == 0) | torch.as_tensor(run.pg_kink[b], device=d.device)).all()
+
+
+# --------------------------------------------------------------------------------------------
+
+def test_tiny_full(oracle):
+    w = inputs.WORKLOADS["tiny"]
+    batch = inputs.make_batch(w, device=DEV)
+    run = OracleRun(oracle, w, batch)
+    out, rep = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    dlogits_properties(run, out, batch["ids"], batch["actor"])
+    # twice the same call: bit-identical results (no atomics on floats, fixed reduction order)
+    out2, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    assert torch.equal(out.loss, out2.loss) and torch.equal(out.dlogits, out2.dlogits)
+
+
+def test_tiny_strided_prompt_view_and_in_place(oracle):
+    # logits of the whole sequence [B,P+T,V]; the response rows are a strided view of it
+    w = inputs.WORKLOADS["tiny"]
+    full = inputs.make_batch(w, device=DEV, with_prompt=True)
+    logits = inputs.response_view(w, full["actor"])
+    ref = inputs.response_view(w, full["ref"])
+    ids = full["ids"][:, w.P:]
+    assert not logits.is_contiguous() and not ids.is_contiguous()
+    run = OracleRun(oracle, w, full, logits_view=logits, ref_view=ref, ids_view=ids)
+    run_steps(oracle, w, full, run, logits, ref, ids, all_rows=True)
+    # in place: dlogits overwrite a copy of the logits (contiguous clone of the view)
+    run_steps(oracle, w, full, run, logits.contiguous(), ref, ids, in_place=True, all_rows=True)
+    # in place on the strided view itself: the prompt rows around it must stay untouched
+    full2 = full["actor"].clone()
+    view2 = inputs.response_view(w, full2)
+    ws = binding.workspace(w.B, w.T, DEV)
+    out = binding.PPOOutputs(view2, in_place=True)
+    binding.ppo_loss_fwd_bwd(view2, ids, full["lengths"], torch.as_tensor(run.lp_old_in, device=DEV),
+                             torch.as_tensor(run.adv_in, device=DEV), torch.as_tensor(run.values_new_in, device=DEV),
+                             torch.as_tensor(run.values_old_in, device=DEV), torch.as_tensor(run.ret_in, device=DEV),
+                             w.clip_eps, w.value_clip, run.grad_scale, ws, out)
+    assert binding.poll_status(ws) == 0
+    assert torch.equal(full2[:, :w.P - 1], full["actor"][:, :w.P - 1])
+    assert torch.equal(full2[:, w.P - 1 + w.T:], full["actor"][:, w.P - 1 + w.T:])
+    check_dlogits_rows(oracle, run, logits, ids, view2, np.arange(w.B * w.T))
+
+
+def test_tiny_special_cases(oracle):
+    w = inputs.WORKLOADS["tiny"]
+    batch = inputs.make_batch(w, device=DEV)
+    # on-policy (rho = 1) and sequence scores outside the reward clip on both sides
+    run = OracleRun(oracle, w, batch, on_policy=True, score_override=np.array([7.5, -9.0], dtype=np.float32))
+    run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    assert (run.ppo.g[run.valid] != 0).all()
+    # grad_scale = 1: the 1/N normalisation is inside the gradient
+    run1 = OracleRun(oracle, w, batch, grad_scale=1.0)
+    run_steps(oracle, w, batch, run1, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    # a wider old-policy spread so that many tokens are clipped (zero-gradient rows)
+    wide = inputs.scaled(w, lp_old_sigma=0.4)
+    bw = inputs.make_batch(wide, device=DEV)
+    runw = OracleRun(oracle, wide, bw)
+    assert (runw.ppo.g[runw.valid] == 0).sum() >= 3
+    run_steps(oracle, wide, bw, runw, bw["actor"], bw["ref"], bw["ids"], all_rows=True)
+
+
+@pytest.mark.parametrize("V", [1000, 1001, 1003, 8, 7, 1, 4099])
+def test_small_odd_vocabularies(oracle, V):
+    # V not a multiple of 8 makes rows that are not 16-byte aligned
+    w = inputs.scaled(inputs.WORKLOADS["tiny"], V=V, B=3, T=9, lengths="uniform:0:9", seed=10 + V)
+    batch = inputs.make_batch(w, device=DEV)
+    run = OracleRun(oracle, w, batch)
+    run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+
+
+def test_ragged_small(oracle):
+    # the ragged recipe (all-pad, length 1 and 2, -inf entries, sharpened rows; gamma .99, lambda 1) at a small size
+    w = inputs.scaled(inputs.WORKLOADS["ragged"], B=12, T=40, V=4096)
+    batch = inputs.make_batch(w, device=DEV)
+    assert (batch["lengths"][:4].cpu() == torch.tensor([0, 1, 2, 40])).all()
+    run = OracleRun(oracle, w, batch)
+    out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    dlogits_properties(run, out, batch["ids"], batch["actor"])
+    # deleted (-inf) entries get a zero gradient
+    dead = torch.isinf(batch["actor"].float())
+    assert dead.any() and (out.dlogits[dead].float() == 0).all()
+
+
+def test_all_padding_batch(oracle):
+    w = inputs.scaled(inputs.WORKLOADS["tiny"], lengths="uniform:0:0")
+    batch = inputs.make_batch(w, device=DEV)
+    assert int(batch["lengths"].sum()) == 0
+    run = OracleRun(oracle, w, batch)
+    out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    assert (out.loss == 0).all() and (out.dlogits.view(torch.int16) == 0).all() and (out.dvalues == 0).all()
+
+
+def test_gae_long_sequences_closed_form(oracle):
+    # T beyond one warp-chunk round, gamma = lambda = 1: returns are reward-to-go (float64 cumsum)
+    rng = np.random.default_rng(5)
+    B, T = 7, 3000
+    lengths = np.array([3000, 2999, 1025, 1024, 33, 1, 0], dtype=np.int32)
+    r = rng.normal(0, 1, (B, T)).astype(np.float32)
+    v = rng.normal(0, 1, (B, T)).astype(np.float32)
+    adv, ret = binding.gae(_t(r), _t(v), _t(lengths, torch.int32), 1.0, 1.0)
+    for b, n in enumerate(lengths):
+        togo = np.cumsum(r[b, :n][::-1].astype(np.float64))[::-1]
+        ok, ratio = close_rel(np32(ret)[b, :n], togo)
+        assert ok, (b, ratio)
+    for gamma, lam in ((0.99, 0.95), (0.9, 1.0), (1.0, 0.0)):
+        adv, ret = binding.gae(_t(r), _t(v), _t(lengths, torch.int32), gamma, lam)
+        wa, wr = oracle.gae(r, v, lengths, gamma, lam)
+        assert close_rel(np32(adv), wa)[0] and close_rel(np32(ret), wr)[0]
