@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the token-level PPO path: response tokens/s and achieved HBM bandwidth.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload opt] [--impl ours|reference]
+
+One step is one pass of the whole path over one synthetic batch that is resident in HBM:
+log-probs of the actor logits and of the reference logits, the KL-penalised reward, GAE, and the
+fused PPO loss forward/backward that writes bf16 dlogits.  The line printed at the end is JSON.
+
+--impl reference times the float64 CPU oracle (plain C, OpenMP over rows) on the host cores on
+the same workload; it is a deliberately slow program, reported as a baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused logprob+PPO fwd/bwd: logit GB/s vs HBM peak; response tokens/s"
+UNIT = "response tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch of the loss kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
+# ncu capture summarised under profiles/, valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {"sources_sha256": None, "workload": None, "bytes_per_launch": None}
+
+
+def sources_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2410_15651_b200", "csrc")
+    for f in sorted(os.listdir(csrc)):
+        h.update(open(os.path.join(csrc, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons of one GPU with nvidia-smi while a region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.out = None
+
+    def start(self):
+        try:
+            self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.flush()
+        rows = [l.strip().split(", ") for l in open(self.out.name) if l.strip()]
+        os.unlink(self.out.name)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.strip().lower() == "active":
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------ CUDA arm
+
+class Path:
+    """All buffers of one step, resident on the device, and the step itself (C-ABI calls only)."""
+
+    def __init__(self, w, batch, dev):
+        import torch
+        from paper_2410_15651_b200 import binding
+        self.b, self.w, self.binding = batch, w, binding
+        B, T = w.B, w.T
+        self.ws = binding.workspace(B, T, dev)
+        f = lambda: torch.empty((B, T), dtype=torch.float32, device=dev)
+        self.lp_act, self.lp_ref, self.rewards, self.adv, self.ret = f(), f(), f(), f(), f()
+        self.out = binding.PPOOutputs(batch["actor"])
+        self.N = int(batch["lengths"].sum().item())
+        # old-policy log-probs = current + N(0, sigma^2) on valid tokens, prepared once outside the timed region
+        cur = binding.gather_logprobs(batch["actor"], batch["ids"], batch["lengths"], self.ws)
+        mask = torch.arange(T, device=dev)[None, :] < batch["lengths"][:, None]
+        self.lp_old = (cur + batch["lp_old_noise"] * mask).contiguous()
+        self.launches_per_step = 6
+
+    def step(self, ev=None):
+        b, w, k = self.b, self.w, self.binding
+        k.gather_logprobs(b["actor"], b["ids"], b["lengths"], self.ws, self.lp_act)
+        k.gather_logprobs(b["ref"], b["ids"], b["lengths"], self.ws, self.lp_ref)
+        k.kl_reward(self.lp_old, self.lp_ref, b["score"], b["lengths"], w.beta_kl, w.reward_clip, self.rewards)
+        k.gae(self.rewards, b["values_old"], b["lengths"], w.gamma, w.lam, self.adv, self.ret)
+        if ev is not None:
+            ev[0].record()
+        k.ppo_loss_fwd_bwd(b["actor"], b["ids"], b["lengths"], self.lp_old, self.adv, b["values_new"],
+                           b["values_old"], self.ret, w.clip_eps, w.value_clip, float(self.N), self.ws, self.out)
+        if ev is not None:
+            ev[1].record()
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2410_15651_b200 import binding, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("launch with torch.distributed.run for --gpus > 1")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    binding.lib()                                              # fail here, loudly, if not built
+    w = inputs.scaled(inputs.WORKLOADS[args.workload], seed=inputs.WORKLOADS[args.workload].seed + 1000 * rank)
+    batch = inputs.make_batch(w, device=dev)
+    path = Path(w, batch, dev)
+    B, T, V = w.B, w.T, w.V
+    n_valid = path.N
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        path.step()
+    assert binding.poll_status(path.ws) == 0
+
+    # ---- device-resident throughput: exactly K steps, CUDA events on the launching stream
+    K = args.steps
+    inner = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sync_all()
+    sampler.start()
+    t0.record()
+    for i in range(K):
+        path.step(inner[i])
+    t1.record()
+    sync_all()
+    clocks = sampler.stop()
+    elapsed_ms = t0.elapsed_time(t1)
+    loss_ms = sum(a.elapsed_time(b) for a, b in inner) / K
+    assert binding.poll_status(path.ws) == 0
+
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+        n = torch.tensor([n_valid], device=dev, dtype=torch.float64)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+        total_tokens = float(n.item())
+    else:
+        total_tokens = float(n_valid)
+    ms_per_step = elapsed_ms / K
+    value = total_tokens / (ms_per_step * 1e-3)
+
+    # ---- end to end: inputs start in pinned host memory, losses are read back, every step
+    host = {k: batch[k].cpu().pin_memory() for k in ("actor", "ref", "ids", "lengths", "values_old",
+                                                      "values_new", "score")}
+    host["lp_old"] = path.lp_old.cpu().pin_memory()
+    loss_host = torch.empty(2, dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = loss_host.numel() * 4
+    e_steps = max(3, min(20, K))
+
+    def e2e_step():
+        for k_ in ("actor", "ref", "ids", "lengths", "values_old", "values_new", "score"):
+            batch[k_].copy_(host[k_], non_blocking=True)
+        path.lp_old.copy_(host["lp_old"], non_blocking=True)
+        path.step()
+        loss_host.copy_(path.out.loss, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e_steps):
+        e2e_step()
+    e1.record()
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = total_tokens / (e2e_ms / e_steps * 1e-3)
+
+    # ---- roofline of the dominant kernel (the loss forward/backward)
+    peak, peak_src = hbm_peak()
+    loss_bytes = 2.0 * V * n_valid + 2.0 * V * B * T          # logits read on valid rows + dlogits written on all rows
+    achieved = loss_bytes / (loss_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["sources_sha256"] == sources_digest() and NCU_TRAFFIC["workload"] == args.workload:
+        traffic = NCU_TRAFFIC["bytes_per_launch"]
+    step_bytes = loss_bytes + 2 * (2.0 * V * n_valid)         # + the two log-prob passes
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: B={B} T={T} V={V} bf16 logits, {n_valid} response tokens per GPU",
+                   "l2": "inputs larger than L2 (%.2f GB touched per step)" % (step_bytes / 1e9 + 0.0),
+                   "multi_gpu": "independent batch per rank, no data-path collective"},
+        "clocks": clocks, "gpu_launches": path.launches_per_step * K,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e_steps},
+        "roofline": {"bound": "hbm", "kernel": "rlhf_ppo_loss_fwd_bwd (row kernel + finalisation)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": peak_src, "traffic": traffic, "ms_per_launch": loss_ms,
+                     "algorithmic_bytes_per_launch": loss_bytes,
+                     "step_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=20.0)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------ oracle arm
+
+def oracle_pass(oracle, w, batch_np, seqs):
+    """The whole path on the CPU oracle for the listed sequences; returns response tokens processed."""
+    import numpy as np
+    sl = np.asarray(seqs)
+    actor, ref, ids = batch_np["actor"][sl], batch_np["ref"][sl], batch_np["ids"][sl]
+    ln = batch_np["lengths"][sl]
+    lp_act = oracle.gather_logprobs(actor, ids, ln)
+    lp_ref = oracle.gather_logprobs(ref, ids, ln)
+    valid = np.arange(w.T)[None, :] < ln[:, None]
+    lp_old = np.where(valid, lp_act + batch_np["lp_old_noise"][sl], 0.0)
+    r = oracle.kl_reward(lp_old, lp_ref, batch_np["score"][sl], ln, w.beta_kl, w.reward_clip)
+    adv, ret = oracle.gae(r, batch_np["values_old"][sl], ln, w.gamma, w.lam)
+    n = int(ln.sum())
+    out = oracle.ppo_loss(actor, ids, ln, lp_old, adv, batch_np["values_new"][sl], batch_np["values_old"][sl],
+                          ret, w.clip_eps, w.value_clip, float(max(n, 1)))
+    for i in range(len(sl)):                                    # dlogits of every row, one sequence at a time
+        rows = np.arange(i * w.T, (i + 1) * w.T)
+        oracle.dlogits_rows(actor, ids, ln, out.g, rows)
+    return n
+
+
+def oracle_inputs(workload: str, n_seq: int):
+    import numpy as np
+    from paper_2410_15651_b200 import inputs
+    w0 = inputs.WORKLOADS[workload]
+    w = inputs.scaled(w0, B=min(w0.B, n_seq))
+    b = inputs.make_batch(w, device="cpu")
+    bn = {k: (inputs.bf16_bits(v) if v.dtype.is_floating_point and v.element_size() == 2 else v.numpy())
+          for k, v in b.items()}
+    bn["lengths"] = bn["lengths"].astype(np.int32)
+    return w, bn
+
+
+def cpu_baseline(workload: str, budget_s: float):
+    """The oracle, as it stands, on a bounded sample of the workload: whole sequences, as many as fit
+    in about `budget_s` seconds of wall time on the host cores."""
+    import oracle
+    oracle.build()
+    w, bn = oracle_inputs(workload, n_seq=2)
+    t0 = time.perf_counter()
+    n = oracle_pass(oracle, w, bn, [0])
+    dt = time.perf_counter() - t0
+    reps = max(1, int(budget_s / max(dt, 1e-3)) // 4)
+    t0 = time.perf_counter()
+    tokens = 0
+    for i in range(reps):
+        tokens += oracle_pass(oracle, w, bn, [i % w.B])
+    dt = time.perf_counter() - t0
+    return {"value": tokens / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{reps} sequence passes of the {workload} workload (T={w.T}, V={w.V}), "
+                      f"{tokens} response tokens, {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    from paper_2410_15651_b200 import inputs
+    w, bn = oracle_inputs(args.workload, n_seq=2)
+    full = inputs.WORKLOADS[args.workload]
+    for i in range(min(args.warmup, 2)):
+        oracle_pass(oracle, w, bn, [0])
+    t0 = time.perf_counter()
+    tokens = 0
+    steps = min(args.steps, 12)                               # each step: one sequence of the workload
+    for i in range(steps):
+        tokens += oracle_pass(oracle, w, bn, [i % w.B])
+    dt = time.perf_counter() - t0
+    value = tokens / dt
+    sample = (f"each step = one sequence of the {args.workload} workload (T={w.T}, V={w.V}); "
+              f"{steps} steps timed, {tokens} response tokens")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": dt / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: B={full.B} T={full.T} V={full.V} bf16 logits (sampled by sequence)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="opt", choices=["tiny", "opt", "llama2", "large_vocab", "ragged"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

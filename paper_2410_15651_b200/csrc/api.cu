@@ -9,6 +9,7 @@
 
 #include "common.cuh"
 #include "kernels_generic.cuh"
+#include "kernels_ring.cuh"
 #include "kernels_small.cuh"
 
 namespace {
@@ -54,7 +55,8 @@ int check_workspace(const void* ws, size_t bytes, int B, int T)
 
 struct DeviceInfo {
     int sm_count = 0;
-    int max_smem_optin = 0;
+    int max_smem_optin = 0;     // per block
+    int smem_per_sm = 0;
 };
 
 // Queried per call: the library keeps no state, and the two attributes are cheap to read.
@@ -64,7 +66,45 @@ int device_info(DeviceInfo& d)
     RLHF_CUDA(cudaGetDevice(&dev));
     RLHF_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
     RLHF_CUDA(cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    RLHF_CUDA(cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
     return RLHF_OK;
+}
+
+// Rows can take the 16-byte path if every row starts on a 16-byte boundary and is a whole number
+// of 16-byte vectors long.
+bool rows_16B(const void* base, long long stride_b, long long stride_t, int V)
+{
+    return aligned(base, 16) && (stride_b % 8) == 0 && (stride_t % 8) == 0 && (V % 8) == 0;
+}
+
+template <bool kLoss, int U>
+int launch_ring_u(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_t s)
+{
+    RLHF_CUDA(cudaFuncSetAttribute(row_ring_kernel<kLoss, U>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)pl.smem_bytes));
+    row_ring_kernel<kLoss, U><<<grid, kRingThreads, pl.smem_bytes, s>>>(ra);
+    return RLHF_OK;
+}
+
+template <bool kLoss>
+int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
+{
+    const unsigned row_bytes = 2u * (unsigned)a.V;
+    const RingPlan pl = plan_ring(row_bytes, kLoss, dev.smem_per_sm, dev.max_smem_optin);
+    RingArgs ra{};
+    ra.row = a;
+    ra.n_slots = pl.n_slots;
+    ra.chunks_per_row = pl.chunks_per_row;
+    ra.resident = pl.resident;
+    ra.row_bytes = row_bytes;
+    const long long rows = (long long)a.B * a.T;
+    const int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * pl.blocks_per_sm);
+    int e = RLHF_OK;
+    switch (pl.U) {
+        case 1: e = launch_ring_u<kLoss, 1>(ra, pl, grid, s); break;
+        default: e = launch_ring_u<kLoss, 2>(ra, pl, grid, s); break;
+    }
+    return e;
 }
 
 int launch_check(const char* what)
@@ -165,6 +205,10 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
     a.status = (unsigned*)workspace;
     a.out_lp = out_logprobs;
 
+    if (rows_16B(logits, stride_b, stride_t, V)) {
+        if (int e = launch_ring<false>(a, dev, (cudaStream_t)stream)) return e;
+        return launch_check("row_ring_kernel<logprob>");
+    }
     long long rows = (long long)B * T;
     int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
     row_generic_kernel<false><<<grid, kGenericThreads, 0, (cudaStream_t)stream>>>(a);
@@ -259,9 +303,14 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
 
     cudaStream_t s = (cudaStream_t)stream;
     long long rows = (long long)B * T;
-    int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
-    row_generic_kernel<true><<<grid, kGenericThreads, 0, s>>>(a);
-    if (int e = launch_check("row_generic_kernel<loss>")) return e;
+    if (rows_16B(logits, stride_b, stride_t, V) && rows_16B(out_dlogits, dl_stride_b, dl_stride_t, V)) {
+        if (int e = launch_ring<true>(a, dev, s)) return e;
+        if (int e = launch_check("row_ring_kernel<loss>")) return e;
+    } else {
+        int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
+        row_generic_kernel<true><<<grid, kGenericThreads, 0, s>>>(a);
+        if (int e = launch_check("row_generic_kernel<loss>")) return e;
+    }
 
     FinalArgs f{};
     f.lengths = lengths;

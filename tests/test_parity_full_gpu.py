@@ -1,0 +1,33 @@
+"""CUDA path against the CPU oracle at the full sizes of the OPT-shaped, Llama-2-shaped,
+large-vocabulary and ragged workloads, in the launch configuration the benchmark times.
+
+Every O(B*T) output (log-probs of all rows for actor and reference, rewards, advantages, returns,
+dvalues, both losses) is compared in full: the oracle computes all of them.  The bf16 logits
+gradient is compared element by element on a sample of rows (valid, padded, zero-gradient, first
+and last), and checked on every row through properties that need no oracle row.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2410_15651_b200 import binding, inputs
+
+from helpers import OracleRun
+from test_parity_gpu import DEV, dlogits_properties, run_steps, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,in_place", [("opt", False), ("opt", True), ("llama2", False),
+                                           ("large_vocab", False), ("ragged", False)])
+def test_full_size(oracle, name, in_place):
+    w = inputs.WORKLOADS[name]
+    batch = inputs.make_batch(w, device=DEV)
+    run = OracleRun(oracle, w, batch)
+    rows = sample_rows(run, 48, seed=w.seed)
+    out, rep = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"],
+                         in_place=in_place, sample_rows=rows)
+    dlogits_properties(run, out, batch["ids"], batch["actor"])
+    print(name, {k: (round(v, 4) if isinstance(v, float) else v) for k, v in rep.items()})
+    del batch, out
+    torch.cuda.empty_cache()
