@@ -61,6 +61,7 @@ typedef enum {
     RLHF_ERR_WORKSPACE = 5,     /* workspace smaller than rlhf_workspace_bytes(B,T) */
     RLHF_ERR_SCALAR = 6,        /* non-finite or out-of-range scalar argument */
     RLHF_ERR_CUDA = 7,          /* a CUDA runtime call or launch failed; see rlhf_last_cuda_error */
+    RLHF_ERR_TOO_LARGE = 8,     /* rlhf_ppo_loss_fwd_bwd_noalloc: B*T above RLHF_NOALLOC_MAX_TOKENS */
     /* device-detected, sticky in the workspace, bit flags (may be OR-ed together) */
     RLHF_ERR_ID_RANGE = 16,     /* a generated-token id outside [0,V) at a valid position */
     RLHF_ERR_LENGTH_RANGE = 32, /* a length outside [0,T] (clamped) */
@@ -162,6 +163,44 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
                           void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
                           float* out_dvalues, float* out_lp_new,
                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Step 4 for callers that cannot provide a workspace.  (The paper has no counterpart to this
+ * entry point; it exists for integration reasons only.)
+ *
+ * Some callers have no way to obtain scratch memory: a plug-in that is handed raw tensor pointers
+ * but no allocator; a process in which a framework's caching allocator has already reserved the
+ * whole device, so that a direct cudaMalloc fails; a latency-critical loop that must not take the
+ * implicit device synchronisation of cudaMalloc/cudaFree.  For them this variant computes exactly
+ * what rlhf_ppo_loss_fwd_bwd computes, with the same arguments minus the workspace, and takes
+ * its scratch from a fixed array that is part of the library image in device memory.
+ *
+ *  - The array holds the scratch for at most RLHF_NOALLOC_MAX_TOKENS = 65536 tokens (B*T); it is
+ *    about 264 KB and is resident on every GPU that loads the library, until the process exits.
+ *    A larger batch is refused with RLHF_ERR_TOO_LARGE and nothing is launched.
+ *  - The call allocates and frees nothing, directly or through any library.
+ *  - The first call on each device looks up the device address of the array (with that device
+ *    current) and remembers it.  Make that first call outside any stream capture.
+ *  - All calls on one device share the array, and it keeps what the previous call left in it.
+ *    The call itself clears the words that must start at zero.  Two calls whose kernels can run
+ *    at the same time on one device (different streams without an ordering between them) race on
+ *    the array and give undefined results: keep calls on one stream, or order them with events.
+ *  - out_device_status: optional device pointer to one 32-bit word; if given, the device-detected
+ *    status flags of this call (RLHF_ERR_ID_RANGE, ...; 0 if none) are copied there on `stream`.
+ *  Everything else (arguments, layouts, aliasing rules, return value) is as for
+ *  rlhf_ppo_loss_fwd_bwd.
+ */
+#define RLHF_NOALLOC_MAX_TOKENS 65536
+
+int rlhf_ppo_loss_fwd_bwd_noalloc(const void* logits, long long stride_b, long long stride_t,
+                                  const long long* ids, long long ids_stride_b, const int* lengths,
+                                  const float* lp_old, const float* adv, const float* values_new,
+                                  const float* values_old, const float* returns,
+                                  int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
+                                  float* out_loss_pg, float* out_loss_vf,
+                                  void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                                  float* out_dvalues, float* out_lp_new,
+                                  unsigned int* out_device_status, void* stream);
 
 #ifdef __cplusplus
 }

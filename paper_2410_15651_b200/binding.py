@@ -34,7 +34,12 @@ SIGNATURES = {
     "rlhf_ppo_loss_fwd_bwd": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
                                      _int, _int, _int, _f32, _f32, _f32, _vp, _vp,
                                      _vp, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
+    "rlhf_ppo_loss_fwd_bwd_noalloc": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
+                                             _int, _int, _int, _f32, _f32, _f32, _vp, _vp,
+                                             _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
 }
+
+NOALLOC_MAX_TOKENS = 65536
 
 _lib = None
 
@@ -218,4 +223,40 @@ def ppo_loss_fwd_bwd(logits: torch.Tensor, ids: torch.Tensor, lengths: torch.Ten
         loss.data_ptr(), loss.data_ptr() + 4,
         out.dlogits.data_ptr(), dsb, dst, out.dvalues.data_ptr(), lp_new_ptr,
         ws.data_ptr(), ws.numel(), _stream(logits)), "rlhf_ppo_loss_fwd_bwd")
+    return out
+
+
+def ppo_loss_fwd_bwd_noalloc(logits: torch.Tensor, ids: torch.Tensor, lengths: torch.Tensor,
+                             lp_old: torch.Tensor, adv: torch.Tensor, values_new: torch.Tensor,
+                             values_old: torch.Tensor, returns: torch.Tensor,
+                             clip_eps: float, value_clip: float, grad_scale: float,
+                             out: PPOOutputs, device_status: Optional[torch.Tensor] = None) -> PPOOutputs:
+    """rlhf_ppo_loss_fwd_bwd_noalloc: the same computation with no workspace argument, for callers
+    that cannot allocate scratch memory (at most NOALLOC_MAX_TOKENS tokens; calls on one device must
+    not overlap).  `out` must be given (this wrapper allocates nothing either); `device_status`,
+    if given, is an int32 CUDA tensor of one element that receives the device-detected flags."""
+    B, T, V, sb, st = _logits(logits, "logits")
+    isb = _ids(ids, B, T)
+    _lengths(lengths, B)
+    for name, t in (("lp_old", lp_old), ("adv", adv), ("values_new", values_new),
+                    ("values_old", values_old), ("returns", returns)):
+        _bt(t, B, T, name)
+    dB, dT, dV, dsb, dst = _logits(out.dlogits, "out.dlogits")
+    if (dB, dT, dV) != (B, T, V):
+        raise ValueError("out.dlogits must have the shape of logits")
+    _bt(out.dvalues, B, T, "out.dvalues")
+    lp_new_ptr = None
+    if out.lp_new is not None:
+        lp_new_ptr = _bt(out.lp_new, B, T, "out.lp_new").data_ptr()
+    loss = _dev(out.loss, torch.float32, "out.loss")
+    st_ptr = None
+    if device_status is not None:
+        st_ptr = _dev(device_status, torch.int32, "device_status").data_ptr()
+    _check(lib().rlhf_ppo_loss_fwd_bwd_noalloc(
+        logits.data_ptr(), sb, st, ids.data_ptr(), isb, lengths.data_ptr(),
+        lp_old.data_ptr(), adv.data_ptr(), values_new.data_ptr(), values_old.data_ptr(), returns.data_ptr(),
+        B, T, V, clip_eps, value_clip, grad_scale,
+        loss.data_ptr(), loss.data_ptr() + 4,
+        out.dlogits.data_ptr(), dsb, dst, out.dvalues.data_ptr(), lp_new_ptr,
+        st_ptr, _stream(logits)), "rlhf_ppo_loss_fwd_bwd_noalloc")
     return out

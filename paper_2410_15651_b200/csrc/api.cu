@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 #include "kernels_generic.cuh"
@@ -129,6 +130,7 @@ const char* rlhf_status_string(int status)
         case RLHF_ERR_WORKSPACE: return "RLHF_ERR_WORKSPACE";
         case RLHF_ERR_SCALAR: return "RLHF_ERR_SCALAR";
         case RLHF_ERR_CUDA: return "RLHF_ERR_CUDA";
+        case RLHF_ERR_TOO_LARGE: return "RLHF_ERR_TOO_LARGE";
         default: break;
     }
     if (status > 0 && (status & ~(RLHF_ERR_ID_RANGE | RLHF_ERR_LENGTH_RANGE | RLHF_ERR_TIMEOUT)) == 0) {
@@ -334,3 +336,66 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Entry point for callers that cannot allocate: scratch lives in a fixed device array of this image.
+constexpr size_t kNoallocScratchBytes = 8192 + 4 * (size_t)RLHF_NOALLOC_MAX_TOKENS;
+
+// In host code this name is only a handle for the symbol, not a device address; the address is
+// obtained per device with cudaGetSymbolAddress below and that pointer is what the kernels get.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocScratchBytes];
+
+namespace {
+
+static_assert(kNoallocScratchBytes == kRowLossOffset + 4 * (size_t)RLHF_NOALLOC_MAX_TOKENS,
+              "scratch array must hold the workspace of RLHF_NOALLOC_MAX_TOKENS tokens");
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device, looked up on first use per device.
+int noalloc_scratch(void** out)
+{
+    int dev = 0;
+    RLHF_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return cuda_fail(cudaErrorInvalidDevice, "device ordinal above 63");
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        RLHF_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        if (!ptr) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress returned a null address");
+        g_noalloc_ptr[dev] = ptr;
+    }
+    *out = g_noalloc_ptr[dev];
+    return RLHF_OK;
+}
+
+}  // namespace
+
+extern "C" int rlhf_ppo_loss_fwd_bwd_noalloc(const void* logits, long long stride_b, long long stride_t,
+                                             const long long* ids, long long ids_stride_b, const int* lengths,
+                                             const float* lp_old, const float* adv, const float* values_new,
+                                             const float* values_old, const float* returns,
+                                             int B, int T, int V, float clip_eps, float value_clip,
+                                             float grad_scale, float* out_loss_pg, float* out_loss_vf,
+                                             void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                                             float* out_dvalues, float* out_lp_new,
+                                             unsigned int* out_device_status, void* stream)
+{
+    if (B <= 0 || T <= 0) return RLHF_ERR_SHAPE;
+    if ((long long)B * (long long)T > (long long)RLHF_NOALLOC_MAX_TOKENS) return RLHF_ERR_TOO_LARGE;
+    if (out_device_status && !aligned(out_device_status, 4)) return RLHF_ERR_ALIGN;
+    void* scratch = nullptr;
+    if (int e = noalloc_scratch(&scratch)) return e;
+    cudaStream_t s = (cudaStream_t)stream;
+    // the status word and the reduction ticket must start at zero; the rest is written before it is read
+    RLHF_CUDA(cudaMemsetAsync(scratch, 0, 8, s));
+    int e = rlhf_ppo_loss_fwd_bwd(logits, stride_b, stride_t, ids, ids_stride_b, lengths, lp_old, adv,
+                                  values_new, values_old, returns, B, T, V, clip_eps, value_clip, grad_scale,
+                                  out_loss_pg, out_loss_vf, out_dlogits, dl_stride_b, dl_stride_t,
+                                  out_dvalues, out_lp_new, scratch, kNoallocScratchBytes, stream);
+    if (e != RLHF_OK) return e;
+    if (out_device_status)
+        RLHF_CUDA(cudaMemcpyAsync(out_device_status, scratch, 4, cudaMemcpyDeviceToDevice, s));
+    return RLHF_OK;
+}
