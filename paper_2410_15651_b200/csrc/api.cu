@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "kernels_generic.cuh"
 #include "kernels_ring.cuh"
+#include "kernels_dbuf.cuh"
 #include "kernels_small.cuh"
 
 namespace {
@@ -78,12 +79,34 @@ bool rows_16B(const void* base, long long stride_b, long long stride_t, int V)
     return aligned(base, 16) && (stride_b % 8) == 0 && (stride_t % 8) == 0 && (V % 8) == 0;
 }
 
-template <bool kLoss, int U>
-int launch_ring_u(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_t s)
+template <bool kLoss, int NW, int U>
+int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_t s)
 {
-    RLHF_CUDA(cudaFuncSetAttribute(row_ring_kernel<kLoss, U>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RLHF_CUDA(cudaFuncSetAttribute(row_ring_kernel<kLoss, NW, U>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)pl.smem_bytes));
-    row_ring_kernel<kLoss, U><<<grid, kRingThreads, pl.smem_bytes, s>>>(ra);
+    row_ring_kernel<kLoss, NW, U><<<grid, NW * 32 + 32, pl.smem_bytes, s>>>(ra);
+    return RLHF_OK;
+}
+
+constexpr int kDbufWarps = 16;
+
+// Loss kernel for rows of which two fit in shared memory; returns false if the row is out of its range.
+bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev)
+{
+    return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes) + 1024 <= (size_t)dev.max_smem_optin;
+}
+
+int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
+{
+    DbufArgs da{};
+    da.row = a;
+    da.row_bytes = 2u * (unsigned)a.V;
+    da.row_stride = (da.row_bytes + 127u) & ~127u;
+    const size_t smem = dbuf_smem_bytes(da.row_bytes);
+    const long long rows = (long long)a.B * a.T;
+    const int grid = (int)std::min<long long>(rows, dev.sm_count);
+    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    loss_dbuf_kernel<kDbufWarps><<<grid, kDbufWarps * 32 + 32, smem, s>>>(da);
     return RLHF_OK;
 }
 
@@ -91,6 +114,9 @@ template <bool kLoss>
 int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 {
     const unsigned row_bytes = 2u * (unsigned)a.V;
+    if constexpr (kLoss) {
+        if (dbuf_applies(row_bytes, dev)) return launch_dbuf(a, dev, s);
+    }
     const RingPlan pl = plan_ring(row_bytes, kLoss, dev.smem_per_sm, dev.max_smem_optin);
     RingArgs ra{};
     ra.row = a;
@@ -100,12 +126,11 @@ int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     ra.row_bytes = row_bytes;
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * pl.blocks_per_sm);
-    int e = RLHF_OK;
-    switch (pl.U) {
-        case 1: e = launch_ring_u<kLoss, 1>(ra, pl, grid, s); break;
-        default: e = launch_ring_u<kLoss, 2>(ra, pl, grid, s); break;
+    if constexpr (kLoss) {
+        if (pl.NW == 16) return launch_ring_as<true, 16, 2>(ra, pl, grid, s);
     }
-    return e;
+    if (pl.U == 1) return launch_ring_as<kLoss, 8, 1>(ra, pl, grid, s);
+    return launch_ring_as<kLoss, 8, 2>(ra, pl, grid, s);
 }
 
 int launch_check(const char* what)

@@ -23,9 +23,6 @@
 
 namespace rlhf {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kRingThreads = kConsumerThreads + 32;
 constexpr int kZeroBytes = 4096;                       // zeroed buffer that feeds the bulk zero-fill
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -102,10 +99,6 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void consumer_barrier()
-{
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
-}
 __device__ __forceinline__ void store_v4(void* p, const uint4& q)
 {
     asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(q.x), "r"(q.y), "r"(q.z), "r"(q.w)
@@ -177,20 +170,92 @@ __device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sig
 __device__ __forceinline__ void patch_label(uint4& o, int j, float value)
 {
     const uint32_t h = pack_bf16x2(value, 0.f) & 0xffffu;
-    uint32_t* w = j < 2 ? &o.x : (j < 4 ? &o.y : (j < 6 ? &o.z : &o.w));
-    *w = (j & 1) ? ((*w & 0x0000ffffu) | (h << 16)) : ((*w & 0xffff0000u) | h);
+    const int ws = j >> 1;
+    uint32_t w = ws == 0 ? o.x : (ws == 1 ? o.y : (ws == 2 ? o.z : o.w));
+    w = (j & 1) ? ((w & 0x0000ffffu) | (h << 16)) : ((w & 0xffff0000u) | h);
+    o.x = ws == 0 ? w : o.x;
+    o.y = ws == 1 ? w : o.y;
+    o.z = ws == 2 ? w : o.z;
+    o.w = ws == 3 ? w : o.w;
+}
+
+// ---------------------------------------------------------------- block-wide merge of partial sums
+// What the owner of the generated token's vector publishes for the row.
+struct LabelInfo {
+    float zy;    // the generated token's logit
+    float ey;    // 2^(x_y - M) against the owner thread's final reference
+    float M;     // that reference
+    float pad;
+};
+
+// Merges the per-thread partial sums of NW consumer warps.  Each warp first agrees on a common
+// reference (max by shuffles), rescales once and adds; lane 0 publishes (M, s); after the consumer
+// barrier the same is done across warps with one partial per lane.  The generated token's own term
+// comes from the LabelInfo its owner thread wrote before the barrier.  Every thread returns the total.
+template <int NW>
+__device__ __forceinline__ Acc consumer_reduce(const Acc& a, float2* s_part, const LabelInfo* s_lab,
+                                               int warp, int lane)
+{
+    float M = a.M;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float s = a.s * ex2(a.M - M);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) s_part[warp] = make_float2(M, s);
+    asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+    const float2 pw = lane < NW ? s_part[lane] : make_float2(kFloorM, 0.f);
+    float Mt = pw.x;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, o));
+    float st = pw.y * ex2(pw.x - Mt);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) st += __shfl_xor_sync(0xffffffffu, st, o);
+    const LabelInfo li = *s_lab;
+    Acc tot;
+    tot.M = fmaxf(Mt, li.M);
+    tot.s = st * ex2(Mt - tot.M);
+    tot.ey = li.ey * ex2(li.M - tot.M);
+    return tot;
 }
 
 // ---------------------------------------------------------------- the kernel
-// Dynamic shared memory: [n_slots * chunk][full barriers n_slots * 8][empty barriers n_slots * 8][zero buffer].
-template <bool kLoss, int U>
-__global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
+// Sum of the exponentials of U vectors against one reference exponent (no range check).
+template <int U>
+__device__ __forceinline__ float exp_sum_vecs(const uint4 (&q)[U], float negM)
 {
-    constexpr uint32_t kChunk = (uint32_t)kConsumerThreads * 16u * U;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        float z[8];
+        unpack8(q[u], z);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i & 3] += ex2(fmaf(z[i], kLog2e, negM));
+    }
+    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+__device__ __forceinline__ float max8_scaled(const uint4& q)
+{
+    float z[8];
+    unpack8(q, z);
+    float m = fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), fmaxf(fmaxf(z[4], z[5]), fmaxf(z[6], z[7])));
+    return fmaxf(m * kLog2e, kFloorM);
+}
+
+// Dynamic shared memory: [n_slots * chunk][full barriers n_slots * 8][empty barriers n_slots * 8][zero buffer].
+// NW consumer warps + 1 producer warp; a chunk is NW*32*U 16-byte vectors.
+template <bool kLoss, int NW, int U>
+__global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) row_ring_kernel(RingArgs ra)
+{
+    constexpr int kCons = NW * 32;
+    constexpr int kThreads = kCons + 32;
+    constexpr uint32_t kChunkVecs = (uint32_t)kCons * U;
+    constexpr uint32_t kChunk = kChunkVecs * 16u;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ long long s_cnt[33];
-    __shared__ Acc s_part[2][kConsumerWarps];
-    __shared__ float s_zy[2];
+    __shared__ float2 s_part[2][32];
+    __shared__ LabelInfo s_lab[2];
 
     const RowArgs& p = ra.row;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -206,19 +271,19 @@ __global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(full_addr + 8u * s, 1);
-            mbar_init(empty_addr + 8u * s, kConsumerWarps);
+            mbar_init(empty_addr + 8u * s, NW);
         }
         fence_mbar_init();
     }
     if (kLoss) {
-        for (int i = tid; i < kZeroBytes / 16; i += kRingThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < kZeroBytes / 16; i += kThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
         fence_async_smem();
     }
     __syncthreads();
 
     bool aborted = false;
 
-    if (warp == kConsumerWarps) {
+    if (warp == NW) {
         // ------------------------------------------------------------ producer
         if (lane != 0) return;
         const long long n_pad = (long long)p.B * p.T - N;
@@ -268,13 +333,14 @@ __global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
     if (!kLoss) {
         // log-prob 0 at padded tokens
         const long long total = (long long)p.B * p.T;
-        for (long long i = (long long)blockIdx.x * kConsumerThreads + tid; i < total; i += G * kConsumerThreads) {
+        for (long long i = (long long)blockIdx.x * kCons + tid; i < total; i += G * kCons) {
             int b = (int)(i / p.T), t = (int)(i % p.T);
             if (t >= clamp_len(__ldg(p.lengths + b), p.T)) p.out_lp[i] = 0.f;
         }
     }
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
     const uint32_t nvec = ra.row_bytes / 16u;
+    const int full_chunks = (int)(nvec / kChunkVecs);          // chunks in which every vector exists
 
     Cursor cur{0, 0};
     int slot = 0;
@@ -306,26 +372,42 @@ __global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
         if (bad_id) { y = 0; if (tid == 0) atomicOr(p.status, kErrIdRange); }
         const uint32_t yvec = (uint32_t)(y >> 3);
         const int yj = (int)(y & 7);
+        const int ychunk = (int)(yvec / kChunkVecs);
 
         const int slot0 = slot;
         const uint32_t phase0 = phase;
 
         // ---- pass 1: partition sum
         Acc a = acc_empty();
+        float zy = 0.f;
+        const bool owner = (yvec % kCons) == (uint32_t)tid;      // this thread sums the generated token's vector
         for (int c = 0; c < chunks; ++c) {
             mbar_wait(full_addr + 8u * slot, phase, p.status, aborted);
-            const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk);
-            const uint32_t v0 = (uint32_t)c * (kConsumerThreads * U) + tid;
-            uint4 q[U];
+            const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk) + tid;
+            if (c < full_chunks && c != ychunk) {
+                // common case: every vector exists and none holds the generated token
+                uint4 q[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (v0 + u * kConsumerThreads < nvec) q[u] = src[u * kConsumerThreads + tid];
+                for (int u = 0; u < U; ++u) q[u] = src[u * kCons];
+                if (c == 0) a.M = max8_scaled(q[0]);               // thread's reference exponent for this row
+                const float vs = exp_sum_vecs<U>(q, -a.M);
+                if (vs <= 1.8446744e19f) {
+                    a.s += vs;
+                } else {
+                    // a logit far above the reference (or a non-finite sum): redo with range handling
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t v = v0 + u * kConsumerThreads;
-                if (v < nvec) {
-                    if (v == yvec) s_zy[par] = acc_add_vec_label(a, q[u], yj);
-                    else acc_add_vec(a, q[u]);
+                    for (int u = 0; u < U; ++u) acc_add_vec(a, q[u]);
+                }
+            } else {
+                const uint32_t v0 = (uint32_t)c * kChunkVecs + tid;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t v = v0 + u * kCons;
+                    if (v < nvec) {
+                        const uint4 q = src[u * kCons];
+                        if (v == yvec) zy = acc_add_vec_label(a, q, yj);
+                        else acc_add_vec(a, q);
+                    }
                 }
             }
             if (!(kLoss && ra.resident)) {
@@ -334,13 +416,9 @@ __global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
             }
             if (++slot == S) { slot = 0; phase ^= 1u; }
         }
-        a = acc_warp_reduce(a);
-        if (lane == 0) s_part[par][warp] = a;
-        consumer_barrier();
-        Acc tot = s_part[par][0];
-#pragma unroll
-        for (int w = 1; w < kConsumerWarps; ++w) tot = acc_merge(tot, s_part[par][w]);
-        const RowResult r = row_finish(tot, s_zy[par]);
+        if (owner) s_lab[par] = LabelInfo{zy, a.ey, a.M, 0.f};
+        const Acc tot = consumer_reduce<NW>(a, s_part[par], &s_lab[par], warp, lane);
+        const RowResult r = row_finish(tot, s_lab[par].zy);
 
         // scalars of the next row, in flight while this row is finished
         fetch_row(k + G);
@@ -359,32 +437,32 @@ __global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
 
         // ---- pass 2: dlogits
         if (ra.resident) { slot = slot0; phase = phase0; }
-        unsigned char* drow = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t);
+        unsigned char* dst = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t) +
+                             (size_t)tid * 16;
         const float c2 = log2f(fabsf(g)) - r.lse2;
         const uint32_t sign2 = g > 0.f ? 0x80008000u : 0u;
         const float dy = g * r.one_m_py;
-        for (int c = 0; c < chunks; ++c) {
+        for (int c = 0; c < chunks; ++c, dst += kChunk) {
             if (!ra.resident) mbar_wait(full_addr + 8u * slot, phase, p.status, aborted);
-            const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk);
-            const uint32_t v0 = (uint32_t)c * (kConsumerThreads * U) + tid;
-            if (g == 0.f) {
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t v = v0 + u * kConsumerThreads;
-                    if (v < nvec) store_v4(drow + (size_t)v * 16, make_uint4(0, 0, 0, 0));
-                }
-            } else {
+            const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk) + tid;
+            if (c < full_chunks && c != ychunk && g != 0.f) {
                 uint4 q[U];
 #pragma unroll
-                for (int u = 0; u < U; ++u)
-                    if (v0 + u * kConsumerThreads < nvec) q[u] = src[u * kConsumerThreads + tid];
+                for (int u = 0; u < U; ++u) q[u] = src[u * kCons];
+#pragma unroll
+                for (int u = 0; u < U; ++u) store_v4(dst + (size_t)u * kCons * 16, grad_vec(q[u], c2, sign2));
+            } else {
+                const uint32_t v0 = (uint32_t)c * kChunkVecs + tid;
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const uint32_t v = v0 + u * kConsumerThreads;
+                    const uint32_t v = v0 + u * kCons;
                     if (v < nvec) {
-                        uint4 o = grad_vec(q[u], c2, sign2);
-                        if (v == yvec) patch_label(o, yj, dy);
-                        store_v4(drow + (size_t)v * 16, o);
+                        uint4 o = make_uint4(0, 0, 0, 0);
+                        if (g != 0.f) {
+                            o = grad_vec(src[u * kCons], c2, sign2);
+                            if (v == yvec) patch_label(o, yj, dy);
+                        }
+                        store_v4(dst + (size_t)u * kCons * 16, o);
                     }
                 }
             }
@@ -397,7 +475,8 @@ __global__ void __launch_bounds__(kRingThreads) row_ring_kernel(RingArgs ra)
 
 // ---------------------------------------------------------------- host-side plan
 struct RingPlan {
-    int U = 0;                 // 16-byte vectors per consumer thread per chunk (1 or 2); 0 = not applicable
+    int NW = 0;                // consumer warps per block (8 or 16); 0 = not applicable
+    int U = 0;                 // 16-byte vectors per consumer thread per chunk (1 or 2)
     int n_slots = 0;
     int chunks_per_row = 0;
     int resident = 0;
@@ -405,46 +484,58 @@ struct RingPlan {
     size_t smem_bytes = 0;
 };
 
-inline size_t ring_smem_bytes(int U, int n_slots, bool loss)
+inline size_t ring_smem_bytes(int NW, int U, int n_slots, bool loss)
 {
-    return (size_t)n_slots * (kConsumerThreads * 16 * U) + (size_t)n_slots * 16 + (loss ? kZeroBytes : 0);
+    return (size_t)n_slots * ((size_t)NW * 32 * 16 * U) + (size_t)n_slots * 16 + (loss ? kZeroBytes : 0);
 }
 
-// Chooses chunk size, ring depth and blocks per SM for rows of `row_bytes`.
+// Chooses block shape, chunk size, ring depth and blocks per SM for rows of `row_bytes`.
 // sm_smem: shared memory per SM; block_smem_max: opt-in maximum per block.  The system reserves
 // 1 KB per resident block.
 inline RingPlan plan_ring(unsigned row_bytes, bool loss, int sm_smem, int block_smem_max)
 {
     constexpr size_t kStatic = 1024;                   // static shared memory of the kernel, rounded up
     constexpr size_t kReserved = 1024;
-    constexpr int kMaxBlocksByThreads = 2048 / kRingThreads;      // 7
-    RingPlan best;
-    if (loss) {
-        // resident if a whole row fits: as many blocks per SM as can hold a row each; among chunk
-        // sizes that reach that count take the largest; the ring then grows into what is left.
-        // 8 KB chunks unless the row is short or 4 KB chunks let one more block fit per SM
+    if (loss && row_bytes >= 32768) {
+        // long rows that fit: one block of 16 consumer warps per SM owns all of its shared memory, in
+        // 16 KB chunks; the ring holds the row being processed plus as much of the next as fits, so
+        // loads keep streaming while a row is reduced.
+        const int NW = 16, U = 2;
+        const size_t chunk = (size_t)NW * 32 * 16 * U;
+        const int chunks = (int)((row_bytes + chunk - 1) / chunk);
+        if (ring_smem_bytes(NW, U, chunks, true) + kStatic <= (size_t)block_smem_max) {
+            int S = chunks;
+            while (ring_smem_bytes(NW, U, S + 1, true) + kStatic <= (size_t)block_smem_max) ++S;
+            return RingPlan{NW, U, S, chunks, 1, 1, ring_smem_bytes(NW, U, S, true)};
+        }
+    } else if (loss) {
+        // short rows: blocks of 8 consumer warps, as many per SM as can hold a row each (at most 7 by
+        // thread count); among chunk sizes that reach that count take the preferred one; the ring then
+        // grows into what is left.
+        constexpr int NW = 8;
+        constexpr int kMaxBlocksByThreads = 2048 / (NW * 32 + 32);
+        RingPlan best;
         const int order[2] = {row_bytes >= 16384 ? 2 : 1, row_bytes >= 16384 ? 1 : 2};
         for (int U : order) {
-            const size_t chunk = (size_t)kConsumerThreads * 16 * U;
+            const size_t chunk = (size_t)NW * 32 * 16 * U;
             const int chunks = (int)((row_bytes + chunk - 1) / chunk);
-            const size_t need = ring_smem_bytes(U, chunks, true) + kStatic;
+            const size_t need = ring_smem_bytes(NW, U, chunks, true) + kStatic;
             if (need > (size_t)block_smem_max) continue;
             int k = (int)std::min<size_t>(kMaxBlocksByThreads, (size_t)sm_smem / (need + kReserved));
-            if (k < 1) continue;
-            if (k <= best.blocks_per_sm) continue;
+            if (k < 1 || k <= best.blocks_per_sm) continue;
             const size_t per_block = std::min<size_t>((size_t)sm_smem / k - kReserved, (size_t)block_smem_max) - kStatic;
             int S = chunks;
-            while (ring_smem_bytes(U, S + 1, true) <= per_block) ++S;
-            best = RingPlan{U, S, chunks, 1, k, ring_smem_bytes(U, S, true)};
+            while (ring_smem_bytes(NW, U, S + 1, true) <= per_block) ++S;
+            best = RingPlan{NW, U, S, chunks, 1, k, ring_smem_bytes(NW, U, S, true)};
         }
-        if (best.U) return best;
+        if (best.NW) return best;
     }
-    // streaming: 4 blocks per SM with about 48 KB in flight each
-    const int U = row_bytes > 4096 ? 2 : 1;
-    const size_t chunk = (size_t)kConsumerThreads * 16 * U;
+    // streaming: 4 blocks of 8 consumer warps per SM with about 48 KB in flight each
+    const int NW = 8, U = row_bytes > 4096 ? 2 : 1;
+    const size_t chunk = (size_t)NW * 32 * 16 * U;
     const int chunks = (int)((row_bytes + chunk - 1) / chunk);
     const int S = (int)((48 * 1024) / chunk);
-    return RingPlan{U, S, chunks, 0, 4, ring_smem_bytes(U, S, loss)};
+    return RingPlan{NW, U, S, chunks, 0, 4, ring_smem_bytes(NW, U, S, loss)};
 }
 
 }  // namespace rlhf
