@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -12,6 +13,7 @@
 #include "kernels_generic.cuh"
 #include "kernels_ring.cuh"
 #include "kernels_dbuf.cuh"
+#include "kernels_warp.cuh"
 #include "kernels_small.cuh"
 
 namespace {
@@ -88,12 +90,36 @@ int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_
     return RLHF_OK;
 }
 
+constexpr int kLogprobWarps = 24;
+
+int launch_warp_logprob(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
+{
+    WarpArgs wa{};
+    wa.row = a;
+    wa.row_bytes = 2u * (unsigned)a.V;
+    const size_t smem = warp_kernel_smem_bytes(kLogprobWarps);
+    const long long rows = (long long)a.B * a.T;
+    const int grid = (int)std::min<long long>(rows, dev.sm_count);
+    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem));
+    logprob_warp_kernel<kLogprobWarps><<<grid, kLogprobWarps * 32, smem, s>>>(wa);
+    return RLHF_OK;
+}
+
 constexpr int kDbufWarps = 16;
 
 // Loss kernel for rows of which two fit in shared memory; returns false if the row is out of its range.
 bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev)
 {
     return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes) + 1024 <= (size_t)dev.max_smem_optin;
+}
+
+template <int NW>
+int launch_dbuf_as(const DbufArgs& da, size_t smem, int grid, cudaStream_t s)
+{
+    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    loss_dbuf_kernel<NW><<<grid, NW * 32 + 32, smem, s>>>(da);
+    return RLHF_OK;
 }
 
 int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
@@ -105,9 +131,9 @@ int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     const size_t smem = dbuf_smem_bytes(da.row_bytes);
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    loss_dbuf_kernel<kDbufWarps><<<grid, kDbufWarps * 32 + 32, smem, s>>>(da);
-    return RLHF_OK;
+    const char* tune = getenv("RLHF_TUNE_DBUF_WARPS");
+    if (tune && atoi(tune) == 24) return launch_dbuf_as<24>(da, smem, grid, s);
+    return launch_dbuf_as<kDbufWarps>(da, smem, grid, s);
 }
 
 template <bool kLoss>
@@ -233,8 +259,8 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
     a.out_lp = out_logprobs;
 
     if (rows_16B(logits, stride_b, stride_t, V)) {
-        if (int e = launch_ring<false>(a, dev, (cudaStream_t)stream)) return e;
-        return launch_check("row_ring_kernel<logprob>");
+        if (int e = launch_warp_logprob(a, dev, (cudaStream_t)stream)) return e;
+        return launch_check("logprob_warp_kernel");
     }
     long long rows = (long long)B * T;
     int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);

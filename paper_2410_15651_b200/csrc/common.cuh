@@ -104,11 +104,31 @@ __device__ __forceinline__ RowResult row_finish(const Acc& a, float zy)
     return r;
 }
 
+__device__ __forceinline__ float lg2(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Same as row_finish with the hardware lg2/rcp (relative error about 2^-22): a short dependent
+// chain, for kernels in which a whole block waits on these scalars once per row.
+__device__ __forceinline__ RowResult row_finish_fast(const Acc& a, float zy)
+{
+    RowResult r;
+    float tot = a.s + a.ey;
+    r.lse2 = a.M + lg2(tot);
+    r.lp = fmaf(-r.lse2, kLn2, zy);
+    r.one_m_py = __fdividef(a.s, tot);
+    return r;
+}
+
 // Clipped-surrogate terms of one token: loss and g = d(grad_scale * loss / N) / d lp_new.
+template <bool kFast = false>
 __device__ __forceinline__ void ppo_token(float lp_new, float lp_old, float A, float clip_eps,
                                           float scale_over_N, float& loss, float& g)
 {
-    float rho = expf(lp_new - lp_old);
+    float rho = kFast ? ex2((lp_new - lp_old) * kLog2e) : expf(lp_new - lp_old);
     float unclipped = -A * rho;
     float clipped = -A * fminf(fmaxf(rho, 1.f - clip_eps), 1.f + clip_eps);
     if (unclipped >= clipped) { loss = unclipped; g = unclipped * scale_over_N; }

@@ -6,11 +6,17 @@
 // out of buffer i&1, the bulk copies of row i+1 into the other buffer are already in flight, having
 // been issued when that buffer was released a whole row-time earlier; so, except for the very
 // first row of a block, consumers never wait for HBM, and DRAM sees each row read once and written
-// once.  Synchronisation is per row, not per chunk: two "landed" mbarriers per buffer (a 4-vector
-// head part so that the first row can start early, and the rest) and one "released" mbarrier.
-// Inside a row every thread runs straight-line blocks of 4 vectors (32 logits) with no per-vector
-// branch: range checks are per block, and only the block that holds the generated token takes the
-// careful path.
+// once.  Pass 2 writes the bf16 gradient over the logits in the shared-memory buffer; the producer
+// thread then drains the buffer to global memory with bulk stores and refills it with the row after
+// next as soon as the drain has read it, so that the block's stores and loads keep flowing while
+// the consumers are already reducing the other buffer.  Synchronisation is per row, not per chunk:
+// two "landed" mbarriers per buffer (a 4-vector head part so that the first row can start early, and
+// the rest) and one "computed" mbarrier that hands the finished buffer back to the producer.
+// The producer also looks up each row's scalars (token id, old log-prob, advantage) and hands them
+// to the consumers through shared memory, so that the consumers' per-row work is the reduction and
+// a short scalar chain only.  Inside a row every thread runs straight-line blocks of 4 vectors
+// (32 logits) with no per-vector branch: range checks are per block, and only the block that holds
+// the generated token takes the careful path.
 #pragma once
 #include "kernels_ring.cuh"
 
@@ -22,10 +28,51 @@ struct DbufArgs {
     unsigned row_stride;    // row_bytes rounded up to 128: distance between the two buffers
 };
 
+// What the producer publishes for each row before it arms the row's first "landed" barrier.
+struct RowInfo {
+    long long flat;         // b*T + t
+    long long dl_offset;    // element offset of the dlogits row
+    int y;                  // generated token (0 if it was out of range)
+    int bad_id;
+    float lp_old;
+    float adv;
+};
+
 inline size_t dbuf_smem_bytes(unsigned row_bytes)
 {
     const size_t stride = ((size_t)row_bytes + 127) & ~(size_t)127;
     return 2 * stride + kZeroBytes + 64;       // + 6 mbarriers
+}
+
+// Block-wide total of the partial sums, as consumer_reduce but with log2(NW) cross-warp steps.
+template <int NW>
+__device__ __forceinline__ Acc dbuf_reduce(const Acc& a, float2* s_part, const LabelInfo* s_lab, int warp, int lane)
+{
+    float M = a.M;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float s = a.s * ex2(a.M - M);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) s_part[warp] = make_float2(M, s);
+    asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+    constexpr int kTop = NW > 16 ? 16 : (NW > 8 ? 8 : 4);
+    const float2 pw = lane < NW ? s_part[lane] : make_float2(kFloorM, 0.f);
+    float Mt = pw.x;
+#pragma unroll
+    for (int o = kTop; o > 0; o >>= 1) Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, o));
+    float st = pw.y * ex2(pw.x - Mt);
+#pragma unroll
+    for (int o = kTop; o > 0; o >>= 1) st += __shfl_xor_sync(0xffffffffu, st, o);
+    // lanes >= 2*kTop did not take part; everyone takes lane 0's result
+    Mt = __shfl_sync(0xffffffffu, Mt, 0);
+    st = __shfl_sync(0xffffffffu, st, 0);
+    const LabelInfo li = *s_lab;
+    Acc tot;
+    tot.M = fmaxf(Mt, li.M);
+    tot.s = st * ex2(Mt - tot.M);
+    tot.ey = li.ey * ex2(li.M - tot.M);
+    return tot;
 }
 
 template <int NW>
@@ -34,19 +81,21 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     constexpr int kCons = NW * 32;
     constexpr int kThreads = kCons + 32;
     constexpr uint32_t kPiece = 16384;           // size of one bulk copy
+    constexpr uint32_t kStep = (uint32_t)kCons * 16u;       // bytes between a thread's consecutive vectors
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ long long s_cnt[33];
     __shared__ float2 s_part[2][32];
     __shared__ LabelInfo s_lab[2];
+    __shared__ RowInfo s_row[2];
 
     const RowArgs& p = da.row;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t buf_addr = smem_u32(smem);
     unsigned char* zero_buf = smem + 2 * (size_t)da.row_stride;
     const uint32_t bar_addr = smem_u32(zero_buf + kZeroBytes);
-    // barriers: landed[buf][part] at bar_addr + 8*(2*buf+part), released[buf] at bar_addr + 32 + 8*buf
+    // barriers: landed[buf][part] at bar_addr + 8*(2*buf+part), computed[buf] at bar_addr + 32 + 8*buf
     auto landed = [&](int buf, int part) { return bar_addr + 8u * (2 * buf + part); };
-    auto released = [&](int buf) { return bar_addr + 32u + 8u * buf; };
+    auto computed = [&](int buf) { return bar_addr + 32u + 8u * buf; };
 
     const uint32_t nvec = da.row_bytes / 16u;
     // head part: the first 4 vectors of every thread, if the row has at least twice that
@@ -58,8 +107,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
 
     if (tid == 0) {
         for (int i = 0; i < 4; ++i) mbar_init(bar_addr + 8u * i, 1);
-        mbar_init(released(0), NW);
-        mbar_init(released(1), NW);
+        mbar_init(computed(0), NW);
+        mbar_init(computed(1), NW);
         fence_mbar_init();
     }
     for (int i = tid; i < kZeroBytes / 16; i += kThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
@@ -84,17 +133,41 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 bulk_store(drow + off, smem_u32(zero_buf), min((uint32_t)kZeroBytes, da.row_bytes - off));
             bulk_commit();
         };
+        // Hands buffer (i&1), holding the finished gradient of this block's i-th row, to the bulk-store
+        // engine and waits until it has been read out of shared memory.
+        unsigned char *drow0 = nullptr, *drow1 = nullptr;       // global rows the two buffers drain to
+        auto drain = [&](long long i) {
+            const int buf = (int)(i & 1);
+            mbar_wait(computed(buf), (uint32_t)(i >> 1) & 1u, p.status, aborted);
+            if (aborted) return;
+            const uint32_t srcb = buf_addr + (uint32_t)buf * da.row_stride;
+            for (uint32_t off = 0; off < da.row_bytes; off += kPiece)
+                bulk_store((buf ? drow1 : drow0) + off, srcb + off, min(kPiece, da.row_bytes - off));
+            bulk_commit();
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        };
         long long i = 0;
         for (long long k = blockIdx.x; k < N && !aborted; k += G, ++i) {
             int b, t;
             if (!cursor_seek_valid(cur, k, p.lengths, p.B, p.T, b, t)) break;
             const unsigned char* row = (const unsigned char*)(p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t);
+            RowInfo ri;
+            ri.flat = (long long)b * p.T + t;
+            ri.dl_offset = (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t;
+            const long long y = __ldg(p.ids + (long long)b * p.ids_stride_b + t);
+            ri.bad_id = (y < 0 || y >= p.V) ? 1 : 0;
+            ri.y = ri.bad_id ? 0 : (int)y;
+            ri.lp_old = __ldg(p.lp_old + ri.flat);
+            ri.adv = __ldg(p.adv + ri.flat);
+            if (ri.bad_id) atomicOr(p.status, kErrIdRange);
             const int buf = (int)(i & 1);
-            const uint32_t use = (uint32_t)(i >> 1) & 1u;            // parity of this use of the buffer
-            mbar_wait(released(buf), use ^ 1u, p.status, aborted);
+            if (i >= 2) drain(i - 2);                                // the buffer's previous row goes out first
             if (aborted) break;
+            if (buf) drow1 = (unsigned char*)(p.dlogits + ri.dl_offset);
+            else drow0 = (unsigned char*)(p.dlogits + ri.dl_offset);
+            s_row[buf] = ri;
             const uint32_t dst = buf_addr + (uint32_t)buf * da.row_stride;
-            mbar_arrive_expect_tx(landed(buf, 0), head_bytes);
+            mbar_arrive_expect_tx(landed(buf, 0), head_bytes);       // release: publishes s_row[buf]
             for (uint32_t off = 0; off < head_bytes; off += kPiece)
                 bulk_load(dst + off, row + off, min(kPiece, head_bytes - off), landed(buf, 0));
             mbar_arrive_expect_tx(landed(buf, 1), da.row_bytes - head_bytes);
@@ -106,6 +179,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
             }
         }
         while (pads_done < pads_mine) { zero_fill_next(); ++pads_done; }
+        // the last two rows
+        for (long long j = i >= 2 ? i - 2 : 0; j < i && !aborted; ++j) drain(j);
         bulk_wait_all();
         return;
     }
@@ -115,35 +190,17 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     const int cnt = (uint32_t)tid < nvec ? (int)((nvec - tid + kCons - 1) / kCons) : 0;   // this thread's vectors
     const int head_cnt = min(cnt, (int)(head_vecs / kCons) + ((uint32_t)tid < head_vecs % kCons ? 1 : 0));
 
-    Cursor cur{0, 0};
-    int nb = 0, nt = 0;
-    long long ny = 0;
-    float n_lp_old = 0.f, n_adv = 0.f;
-    auto fetch_row = [&](long long k) {
-        if (k < N && cursor_seek_valid(cur, k, p.lengths, p.B, p.T, nb, nt)) {
-            ny = __ldg(p.ids + (long long)nb * p.ids_stride_b + nt);
-            const long long f = (long long)nb * p.T + nt;
-            n_lp_old = __ldg(p.lp_old + f);
-            n_adv = __ldg(p.adv + f);
-        }
-    };
-    fetch_row(blockIdx.x);
-
     long long i = 0;
     for (long long k = blockIdx.x; k < N; k += G, ++i) {
-        const int b = nb, t = nt;
-        long long y = ny;
-        const float lp_old = n_lp_old, adv = n_adv;
-        const long long flat = (long long)b * p.T + t;
-        const bool bad_id = (y < 0 || y >= p.V);
-        if (bad_id) { y = 0; if (tid == 0) atomicOr(p.status, kErrIdRange); }
-        const uint32_t yvec = (uint32_t)(y >> 3);
-        const int yj = (int)(y & 7);
-        const bool owner = (yvec % kCons) == (uint32_t)tid;
-        const int jy = owner ? (int)(yvec / kCons) : -1;            // which of this thread's vectors holds the label
-
         const int buf = (int)(i & 1), par = buf;
         const uint32_t use = (uint32_t)(i >> 1) & 1u;
+        mbar_wait(landed(buf, 0), use, p.status, aborted);
+        RowInfo ri = s_row[buf];
+        if (aborted) { ri.y = 0; ri.bad_id = 1; ri.flat = 0; }      // stale row info: touch nothing
+        const uint32_t yvec = (uint32_t)ri.y >> 3;
+        const int yj = ri.y & 7;
+        const bool owner = (yvec % kCons) == (uint32_t)tid;
+        const int jy = owner ? (int)(yvec / kCons) : -1;            // which of this thread's vectors holds the label
         const uint4* src = (const uint4*)(smem + (size_t)buf * da.row_stride) + tid;
 
         // ---- pass 1: partition sum
@@ -155,7 +212,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 uint4 q[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) q[u] = src[(size_t)(j + u) * kCons];
-                if (jy >= j && jy < j + 4) {
+                if ((unsigned)(jy - j) < 4u) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         if (j + u == jy) zy = acc_add_vec_label(a, q[u], yj);
@@ -177,32 +234,28 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 else acc_add_vec(a, q);
             }
         };
-        mbar_wait(landed(buf, 0), use, p.status, aborted);
         if (cnt > 0 && jy != 0) a.M = max8_scaled(src[0]);          // this thread's reference exponent for the row
         sum_range(0, head_cnt);
         mbar_wait(landed(buf, 1), use, p.status, aborted);
         sum_range(head_cnt, cnt);
 
         if (owner) s_lab[par] = LabelInfo{zy, a.ey, a.M, 0.f};
-        const Acc tot = consumer_reduce<NW>(a, s_part[par], &s_lab[par], warp, lane);
-        const RowResult r = row_finish(tot, s_lab[par].zy);
-
-        fetch_row(k + G);                                           // next row's scalars, in flight during pass 2
+        const Acc tot = dbuf_reduce<NW>(a, s_part[par], &s_lab[par], warp, lane);
+        const RowResult r = row_finish_fast(tot, s_lab[par].zy);
 
         float loss = 0.f, g = 0.f;
-        if (!bad_id) ppo_token(r.lp, lp_old, adv, p.clip_eps, scale_over_N, loss, g);
-        if (tid == 0) {
-            p.row_loss[flat] = loss;
-            if (p.out_lp_new) p.out_lp_new[flat] = bad_id ? 0.f : r.lp;
+        if (!ri.bad_id) ppo_token<true>(r.lp, ri.lp_old, ri.adv, p.clip_eps, scale_over_N, loss, g);
+        if (tid == 0 && !aborted) {
+            p.row_loss[ri.flat] = loss;
+            if (p.out_lp_new) p.out_lp_new[ri.flat] = ri.bad_id ? 0.f : r.lp;
         }
 
-        // ---- pass 2: dlogits from the resident row
-        unsigned char* dst = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t) +
-                             (size_t)tid * 16;
+        // ---- pass 2: the gradient overwrites the logits in the buffer
+        uint4* dst = (uint4*)(smem + (size_t)buf * da.row_stride) + tid;
         if (g == 0.f) {
-            for (int j = 0; j < cnt; ++j) store_v4(dst + (size_t)j * kCons * 16, make_uint4(0, 0, 0, 0));
+            for (int j = 0; j < cnt; ++j) dst[(size_t)j * kCons] = make_uint4(0, 0, 0, 0);
         } else {
-            const float c2 = log2f(fabsf(g)) - r.lse2;
+            const float c2 = lg2(fabsf(g)) - r.lse2;
             const uint32_t sign2 = g > 0.f ? 0x80008000u : 0u;
             const float dy = g * r.one_m_py;
             int j = 0;
@@ -213,22 +266,23 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 uint4 o[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) o[u] = grad_vec(q[u], c2, sign2);
-                if (jy >= j && jy < j + 4) {
+                if ((unsigned)(jy - j) < 4u) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
                         if (j + u == jy) patch_label(o[u], yj, dy);
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) store_v4(dst + (size_t)(j + u) * kCons * 16, o[u]);
+                for (int u = 0; u < 4; ++u) dst[(size_t)(j + u) * kCons] = o[u];
             }
             for (; j < cnt; ++j) {
                 uint4 o = grad_vec(src[(size_t)j * kCons], c2, sign2);
                 if (j == jy) patch_label(o, yj, dy);
-                store_v4(dst + (size_t)j * kCons * 16, o);
+                dst[(size_t)j * kCons] = o;
             }
         }
+        fence_async_smem();                                         // this thread's writes, before the bulk store reads them
         __syncwarp();
-        if (lane == 0) mbar_arrive(released(buf));
+        if (lane == 0) mbar_arrive(computed(buf));
     }
 }
 

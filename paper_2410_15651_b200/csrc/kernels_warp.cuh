@@ -1,0 +1,188 @@
+// Log-prob kernel for 16-byte aligned rows: one warp per row, no block-level synchronisation.
+//
+// Every warp streams its own rows through a private two-slot ring in shared memory: lane 0 issues
+// the bulk asynchronous copies (4 KB chunks, one mbarrier per slot) and runs two chunks ahead of the
+// warp, across row boundaries; all 32 lanes sum the chunk that has landed.  The per-row reduction is
+// a handful of shuffles inside the warp, so no warp ever waits for another one: while one warp
+// finishes a row the others keep the special-function unit and the memory pipe busy.  With 24 warps
+// per SM about 190 KB of loads are in flight per SM, and short batches (fewer rows than warps)
+// still spread evenly: every row is in flight at once.
+#pragma once
+#include "kernels_ring.cuh"
+
+namespace rlhf {
+
+constexpr int kWarpChunk = 4096;                  // bytes per bulk copy
+constexpr int kWarpSlots = 2;
+constexpr int kWarpChunkVecs = kWarpChunk / 16;   // 256 vectors: 8 per lane
+
+// 32-bit walk over the valid tokens (B*T is at most 2^30): b and the number of valid tokens before b.
+struct Cursor32 {
+    int b;
+    int acc;
+};
+__device__ __forceinline__ bool cursor32_seek(Cursor32& c, int k, const int* __restrict__ lengths, int B, int T,
+                                              int& b, int& t)
+{
+    while (c.b < B) {
+        const int len = clamp_len(__ldg(lengths + c.b), T);
+        if (k < c.acc + len) { b = c.b; t = k - c.acc; return true; }
+        c.acc += len;
+        ++c.b;
+    }
+    return false;
+}
+
+struct WarpArgs {
+    RowArgs row;
+    unsigned row_bytes;     // 2*V, multiple of 16
+};
+
+inline size_t warp_kernel_smem_bytes(int warps_per_block)
+{
+    return (size_t)warps_per_block * (kWarpSlots * kWarpChunk + kWarpSlots * 8);
+}
+
+template <int WPB>
+__global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ long long s_cnt[33];
+
+    const RowArgs& p = wa.row;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    unsigned char* ring = smem + (size_t)warp * (kWarpSlots * kWarpChunk);
+    const uint32_t ring_addr = smem_u32(ring);
+    const uint32_t bar_addr = smem_u32(smem + (size_t)WPB * (kWarpSlots * kWarpChunk)) + (uint32_t)warp * (kWarpSlots * 8);
+
+    const int N = (int)block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
+    if (lane == 0) {
+        for (int s = 0; s < kWarpSlots; ++s) mbar_init(bar_addr + 8u * s, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    // log-prob 0 at padded tokens
+    {
+        const long long total = (long long)p.B * p.T;
+        for (long long i = (long long)blockIdx.x * blockDim.x + tid; i < total; i += (long long)gridDim.x * blockDim.x) {
+            int b = (int)(i / p.T), t = (int)(i % p.T);
+            if (t >= clamp_len(__ldg(p.lengths + b), p.T)) p.out_lp[i] = 0.f;
+        }
+    }
+
+    // rows are dealt to blocks first, then to warps: consecutive rows go to different SMs, and a batch
+    // with fewer rows than warps still loads every SM equally
+    const int gw = warp * (int)gridDim.x + (int)blockIdx.x;       // this warp's first row
+    const int GW = (int)gridDim.x * WPB;
+    const uint32_t nvec = wa.row_bytes / 16u;
+    const int nchunks = (int)((wa.row_bytes + kWarpChunk - 1) / kWarpChunk);
+    const int full_chunks = (int)(wa.row_bytes / kWarpChunk);
+
+    // ---- issue side (lane 0 only uses it): next chunk to request
+    Cursor32 icur{0, 0};
+    int ik = gw;          // row of the next chunk to request
+    int ic = 0;                 // its chunk index
+    int islot = 0;
+    const unsigned char* irow = nullptr;
+    auto issue_seek = [&]() {
+        int b, t;
+        if (ik < N && cursor32_seek(icur, ik, p.lengths, p.B, p.T, b, t))
+            irow = (const unsigned char*)(p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t);
+        else
+            ik = N;
+    };
+    auto issue_next = [&]() {
+        if (ik >= N) return;
+        const uint32_t off = (uint32_t)ic * kWarpChunk;
+        const uint32_t bytes = min((uint32_t)kWarpChunk, wa.row_bytes - off);
+        mbar_arrive_expect_tx(bar_addr + 8u * islot, bytes);
+        bulk_load(ring_addr + (uint32_t)islot * kWarpChunk, irow + off, bytes, bar_addr + 8u * islot);
+        islot = islot + 1 == kWarpSlots ? 0 : islot + 1;
+        if (++ic == nchunks) { ic = 0; ik += GW; issue_seek(); }
+    };
+    if (lane == 0) {
+        issue_seek();
+        for (int s = 0; s < kWarpSlots; ++s) issue_next();
+    }
+
+    // ---- consume side
+    Cursor32 cur{0, 0};
+    bool aborted = false;
+    int slot = 0;
+    uint32_t phases = 0;        // bit s: parity to wait for on slot s
+    int nb = 0, nt = 0;
+    long long ny = 0;
+    auto fetch_row = [&](int k) {
+        if (k < N && cursor32_seek(cur, k, p.lengths, p.B, p.T, nb, nt))
+            ny = __ldg(p.ids + (long long)nb * p.ids_stride_b + nt);
+    };
+    fetch_row(gw);
+
+    for (int k = gw; k < N; k += GW) {
+        const int flat = nb * p.T + nt;
+        long long y = ny;
+        const bool bad_id = (y < 0 || y >= p.V);
+        if (bad_id) { y = 0; if (lane == 0) atomicOr(p.status, kErrIdRange); }
+        const uint32_t yvec = (uint32_t)(y >> 3);
+        const int yj = (int)(y & 7);
+        const int ychunk = (int)(yvec / kWarpChunkVecs);
+        fetch_row(k + GW);                                          // next row's token id, in flight during this row
+
+        Acc a = acc_empty();
+        float zy = 0.f;
+        for (int c = 0; c < nchunks; ++c) {
+            mbar_wait(bar_addr + 8u * slot, (phases >> slot) & 1u, p.status, aborted);
+            phases ^= 1u << slot;
+            const uint4* src = (const uint4*)(ring + (size_t)slot * kWarpChunk) + lane;
+            if (c < full_chunks && c != ychunk) {
+                if (c == 0) a.M = max8_scaled(src[0]);             // this lane's reference exponent for the row
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint4 q[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) q[u] = src[(4 * h + u) * 32];
+                    const float vs = exp_sum_vecs<4>(q, -a.M);
+                    if (vs <= 1.8446744e19f) {
+                        a.s += vs;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) acc_add_vec(a, q[u]);
+                    }
+                }
+            } else {
+                const uint32_t v0 = (uint32_t)c * kWarpChunkVecs + lane;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t v = v0 + u * 32;
+                    if (v < nvec) {
+                        const uint4 q = src[u * 32];
+                        if (v == yvec) zy = acc_add_vec_label(a, q, yj);
+                        else acc_add_vec(a, q);
+                    }
+                }
+            }
+            __syncwarp();                                           // every lane is done with the slot
+            if (lane == 0) issue_next();
+            slot = slot + 1 == kWarpSlots ? 0 : slot + 1;
+        }
+
+        // warp-wide total: common reference, one rescale, sums by shuffle; the label's owner lane broadcasts its term
+        float M = a.M;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        const float sc = ex2(a.M - M);
+        float s = a.s * sc;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const int owner = (int)(yvec & 31u);
+        const float ey = __shfl_sync(0xffffffffu, a.ey * sc, owner);
+        zy = __shfl_sync(0xffffffffu, zy, owner);
+        if (lane == 0 && !aborted) {
+            const RowResult r = row_finish(Acc{M, s, ey}, zy);
+            p.out_lp[flat] = bad_id ? 0.f : r.lp;
+        }
+    }
+}
+
+}  // namespace rlhf
