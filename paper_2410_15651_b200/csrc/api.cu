@@ -159,6 +159,16 @@ int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     return launch_ring_as<kLoss, 8, 2>(ra, pl, grid, s);
 }
 
+// The row kernels run with the largest shared-memory carve-out.  A kernel that prefers another
+// split makes the SMs switch configuration before and after it, which costs microseconds per
+// launch; so the small kernels between them ask for the same carve-out.
+template <typename K>
+int keep_max_carveout(K kernel)
+{
+    RLHF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    return RLHF_OK;
+}
+
 int launch_check(const char* what)
 {
     cudaError_t e = cudaGetLastError();
@@ -280,6 +290,7 @@ int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score,
         return RLHF_ERR_ALIGN;
     long long total = (long long)B * T;
     int grid = (int)std::min<long long>((total + 255) / 256, 1184);
+    if (int e = keep_max_carveout(kl_reward_kernel)) return e;
     kl_reward_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(lp_old, lp_ref, score, lengths, B, T,
                                                            beta_kl, reward_clip, out_rewards);
     return launch_check("kl_reward_kernel");
@@ -298,6 +309,7 @@ int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, 
         out_returns == values_old || out_adv == out_returns)
         return RLHF_ERR_STRIDE;
     int grid = (B + kGaeWarpsPerBlock - 1) / kGaeWarpsPerBlock;
+    if (int e = keep_max_carveout(gae_kernel)) return e;
     gae_kernel<<<grid, kGaeWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(rewards, values_old, lengths, B, T,
                                                                        gamma, lambda, out_adv, out_returns);
     return launch_check("gae_kernel");
@@ -382,6 +394,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
     f.ticket = (unsigned*)(ws + 4);
     f.partials = (double*)(ws + kPartialsOffset);
     int fgrid = (int)std::min<long long>((rows + 1023) / 1024, kFinalMaxBlocks);
+    if (int e = keep_max_carveout(ppo_finalize_kernel)) return e;
     ppo_finalize_kernel<<<fgrid, kFinalThreads, 0, s>>>(f);
     return launch_check("ppo_finalize_kernel");
 }

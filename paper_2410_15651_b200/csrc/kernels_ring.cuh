@@ -530,7 +530,18 @@ inline RingPlan plan_ring(unsigned row_bytes, bool loss, int sm_smem, int block_
         }
         if (best.NW) return best;
     }
-    // streaming: 4 blocks of 8 consumer warps per SM with about 48 KB in flight each
+    if (loss) {
+        // rows larger than shared memory are streamed twice.  One block of 16 consumer warps per SM
+        // keeps the number of rows in flight at the number of SMs, so that the second read of a row
+        // (a few tens of microseconds after the first) is still served by L2.
+        const int NW = 16, U = 2;
+        const size_t chunk = (size_t)NW * 32 * 16 * U;
+        const int chunks = (int)((row_bytes + chunk - 1) / chunk);
+        int S = 2;
+        while (ring_smem_bytes(NW, U, S + 1, true) + kStatic <= (size_t)block_smem_max) ++S;
+        return RingPlan{NW, U, S, chunks, 0, 1, ring_smem_bytes(NW, U, S, true)};
+    }
+    // log-prob streaming (not used by the warp-per-row kernel): 4 blocks of 8 consumer warps per SM
     const int NW = 8, U = row_bytes > 4096 ? 2 : 1;
     const size_t chunk = (size_t)NW * 32 * 16 * U;
     const int chunks = (int)((row_bytes + chunk - 1) / chunk);
