@@ -176,7 +176,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
  * its scratch from a fixed array that is part of the library image in device memory.
  *
  *  - The array holds the scratch for at most RLHF_NOALLOC_MAX_TOKENS = 65536 tokens (B*T); it is
- *    about 264 KB and is resident on every GPU that loads the library, until the process exits.
+ *    about 280 KB and is resident on every GPU that loads the library, until the process exits.
  *    A larger batch is refused with RLHF_ERR_TOO_LARGE and nothing is launched.
  *  - The call allocates and frees nothing, directly or through any library.
  *  - The first call on each device looks up the device address of the array (with that device

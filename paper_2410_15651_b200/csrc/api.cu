@@ -34,11 +34,12 @@ int cuda_fail(cudaError_t e, const char* what)
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
-// Workspace layout (bytes): [0,4) status flags, [4,8) finalisation ticket, [256, 256+4096) block
-// partials of the finalisation (256 blocks x 2 doubles), [kRowLossOffset, +4*B*T) per-token policy
-// loss terms.
+// Workspace layout (bytes): [0,4) status flags, [4,8) finalisation ticket, [256, kRowLossOffset) block
+// partial sums of the two losses (2 doubles per block of the kernel that reduces them),
+// [kRowLossOffset, +4*B*T) per-token policy loss terms (kernels without the fused finalisation).
 constexpr size_t kPartialsOffset = 256;
-constexpr size_t kRowLossOffset = 8192;
+constexpr size_t kRowLossOffset = 24576;
+constexpr int kMaxFusedBlocks = (int)((kRowLossOffset - kPartialsOffset) / 16);   // block partials that fit the header
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -111,7 +112,7 @@ constexpr int kDbufWarps = 16;
 // Loss kernel for rows of which two fit in shared memory; returns false if the row is out of its range.
 bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev)
 {
-    return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes) + 1024 <= (size_t)dev.max_smem_optin;
+    return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes) + 1280 <= (size_t)dev.max_smem_optin;
 }
 
 template <int NW>
@@ -368,9 +369,21 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
 
     cudaStream_t s = (cudaStream_t)stream;
     long long rows = (long long)B * T;
-    if (rows_16B(logits, stride_b, stride_t, V) && rows_16B(out_dlogits, dl_stride_b, dl_stride_t, V)) {
+    if (rows_16B(logits, stride_b, stride_t, V) && rows_16B(out_dlogits, dl_stride_b, dl_stride_t, V) &&
+        dev.sm_count * 7 <= kMaxFusedBlocks) {
+        // fast path: the row kernel also does the finalisation (value loss, dvalues, loss reduction)
+        a.fused = 1;
+        a.values_new = values_new;
+        a.values_old = values_old;
+        a.returns = returns;
+        a.value_clip = value_clip;
+        a.out_dvalues = out_dvalues;
+        a.out_loss_pg = out_loss_pg;
+        a.out_loss_vf = out_loss_vf;
+        a.ticket = (unsigned*)(ws + 4);
+        a.partials = (double*)(ws + kPartialsOffset);
         if (int e = launch_ring<true>(a, dev, s)) return e;
-        if (int e = launch_check("row_ring_kernel<loss>")) return e;
+        return launch_check("loss row kernel");
     } else {
         int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
         row_generic_kernel<true><<<grid, kGenericThreads, 0, s>>>(a);
@@ -403,7 +416,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
 
 // ------------------------------------------------------------------------------------------------
 // Entry point for callers that cannot allocate: scratch lives in a fixed device array of this image.
-constexpr size_t kNoallocScratchBytes = 8192 + 4 * (size_t)RLHF_NOALLOC_MAX_TOKENS;
+constexpr size_t kNoallocScratchBytes = 24576 + 4 * (size_t)RLHF_NOALLOC_MAX_TOKENS;
 
 // In host code this name is only a handle for the symbol, not a device address; the address is
 // obtained per device with cudaGetSymbolAddress below and that pointer is what the kernels get.

@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     __shared__ float2 s_part[2][32];
     __shared__ LabelInfo s_lab[2];
     __shared__ RowInfo s_row[2];
+    __shared__ double s_dbl[32];
 
     const RowArgs& p = da.row;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -189,6 +190,9 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
     const int cnt = (uint32_t)tid < nvec ? (int)((nvec - tid + kCons - 1) / kCons) : 0;   // this thread's vectors
     const int head_cnt = min(cnt, (int)(head_vecs / kCons) + ((uint32_t)tid < head_vecs % kCons ? 1 : 0));
+    // the block's slice of the value loss, while its first row is still on the way (thread 0 keeps the sums)
+    double sum_pg = 0.0, sum_vf = 0.0;
+    if (p.fused) sum_vf = consumer_sum_double<NW>(value_loss_slice(p, N, tid, kCons), s_dbl, warp, lane);
 
     long long i = 0;
     for (long long k = blockIdx.x; k < N; k += G, ++i) {
@@ -246,7 +250,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         float loss = 0.f, g = 0.f;
         if (!ri.bad_id) ppo_token<true>(r.lp, ri.lp_old, ri.adv, p.clip_eps, scale_over_N, loss, g);
         if (tid == 0 && !aborted) {
-            p.row_loss[ri.flat] = loss;
+            if (p.fused) sum_pg += (double)loss; else p.row_loss[ri.flat] = loss;
             if (p.out_lp_new) p.out_lp_new[ri.flat] = ri.bad_id ? 0.f : r.lp;
         }
 
@@ -284,6 +288,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         __syncwarp();
         if (lane == 0) mbar_arrive(computed(buf));
     }
+    if (p.fused && tid == 0) publish_block_losses(p, N, sum_pg, sum_vf);
 }
 
 }  // namespace rlhf

@@ -26,6 +26,17 @@ struct RowArgs {
     long long dl_stride_b, dl_stride_t;
     float* row_loss;            // workspace: per-token policy loss term
     float* out_lp_new;          // optional
+    // step 4, finalisation fused into the row kernel (fused != 0): value loss, dvalues and both scalar losses
+    int fused;
+    const float* values_new;
+    const float* values_old;
+    const float* returns;
+    float value_clip;
+    float* out_dvalues;
+    float* out_loss_pg;
+    float* out_loss_vf;
+    unsigned* ticket;           // workspace word 1, zero between calls
+    double* partials;           // workspace: [gridDim.x][2] block partial sums (policy, value)
 };
 
 constexpr int kGenericThreads = 256;

@@ -20,6 +20,7 @@
 #pragma once
 #include "common.cuh"
 #include "kernels_generic.cuh"
+#include "kernels_small.cuh"
 
 namespace rlhf {
 
@@ -256,6 +257,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
     __shared__ long long s_cnt[33];
     __shared__ float2 s_part[2][32];
     __shared__ LabelInfo s_lab[2];
+    __shared__ double s_dbl[32];
 
     const RowArgs& p = ra.row;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -341,6 +343,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
     const uint32_t nvec = ra.row_bytes / 16u;
     const int full_chunks = (int)(nvec / kChunkVecs);          // chunks in which every vector exists
+    double sum_pg = 0.0, sum_vf = 0.0;                         // block partial sums (thread 0)
+    if (kLoss && p.fused) sum_vf = consumer_sum_double<NW>(value_loss_slice(p, N, tid, kCons), s_dbl, warp, lane);
 
     Cursor cur{0, 0};
     int slot = 0;
@@ -431,7 +435,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
         float loss = 0.f, g = 0.f;
         if (!bad_id) ppo_token(r.lp, lp_old, adv, p.clip_eps, scale_over_N, loss, g);
         if (tid == 0) {
-            p.row_loss[flat] = loss;
+            if (p.fused) sum_pg += (double)loss; else p.row_loss[flat] = loss;
             if (p.out_lp_new) p.out_lp_new[flat] = bad_id ? 0.f : r.lp;
         }
 
@@ -471,6 +475,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
             if (++slot == S) { slot = 0; phase ^= 1u; }
         }
     }
+    if (kLoss && p.fused && tid == 0) publish_block_losses(p, N, sum_pg, sum_vf);
 }
 
 // ---------------------------------------------------------------- host-side plan
@@ -494,7 +499,7 @@ inline size_t ring_smem_bytes(int NW, int U, int n_slots, bool loss)
 // 1 KB per resident block.
 inline RingPlan plan_ring(unsigned row_bytes, bool loss, int sm_smem, int block_smem_max)
 {
-    constexpr size_t kStatic = 1024;                   // static shared memory of the kernel, rounded up
+    constexpr size_t kStatic = 1280;                   // static shared memory of the kernel, rounded up
     constexpr size_t kReserved = 1024;
     if (loss && row_bytes >= 32768) {
         // long rows that fit: one block of 16 consumer warps per SM owns all of its shared memory, in

@@ -2,6 +2,7 @@
 // (value loss, dvalues, deterministic reduction of both losses).
 #pragma once
 #include "common.cuh"
+#include "kernels_generic.cuh"
 
 namespace rlhf {
 
@@ -158,6 +159,74 @@ __global__ void __launch_bounds__(kFinalThreads) ppo_finalize_kernel(FinalArgs p
     }
     __syncthreads();
     if (s_last && threadIdx.x == 0) {
+        __threadfence();
+        double a = 0.0, c = 0.0;
+        for (unsigned k = 0; k < gridDim.x; ++k) {
+            a += ((volatile double*)p.partials)[2 * k];
+            c += ((volatile double*)p.partials)[2 * k + 1];
+        }
+        *p.out_loss_pg = N > 0 ? (float)(a / (double)N) : 0.f;
+        *p.out_loss_vf = N > 0 ? (float)(c / (double)N) : 0.f;
+        *p.ticket = 0u;
+    }
+}
+
+// ---------------------------------------------------------------- step 4: finalisation inside a row kernel
+// The same work as ppo_finalize_kernel, done by the row kernel's own blocks: each block takes a
+// contiguous slice of the B*T tokens for the value loss (at its start, while its first row is still
+// in flight) and sums the policy-loss terms of the rows it processes in the order it processes them
+// (the row assignment is static); the last block to finish adds the block partials in index order.
+// The value-loss part: one thread's share of the block's slice; writes dvalues (and zeroes lp_new at
+// padding) and returns the thread's partial sum of loss terms.
+__device__ inline double value_loss_slice(const RowArgs& p, long long N, int tid, int nthreads)
+{
+    const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
+    const long long total = (long long)p.B * p.T;
+    const long long per_block = (total + gridDim.x - 1) / gridDim.x;
+    const long long begin = per_block * blockIdx.x, end = min(total, begin + per_block);
+    double sum_vf = 0.0;
+    for (long long i = begin + tid; i < end; i += nthreads) {
+        int b = (int)(i / p.T), t = (int)(i % p.T);
+        float dv = 0.f;
+        if (t < clamp_len(__ldg(p.lengths + b), p.T)) {
+            float v = p.values_new[i], vo = p.values_old[i], G = p.returns[i];
+            float vc = vo + fminf(fmaxf(v - vo, -p.value_clip), p.value_clip);
+            float e1 = (v - G) * (v - G), e2 = (vc - G) * (vc - G);
+            if (e1 >= e2) { sum_vf += 0.5 * (double)e1; dv = (v - G) * scale_over_N; }
+            else sum_vf += 0.5 * (double)e2;
+        } else if (p.out_lp_new) {
+            p.out_lp_new[i] = 0.f;
+        }
+        p.out_dvalues[i] = dv;
+    }
+    return sum_vf;
+}
+
+// Sum of one double per consumer thread over NW warps (fixed shuffle tree, then warps in index order).
+// Uses named barrier 1 with NW*32 threads; s_dbl holds 32 doubles.  Thread 0 gets the total.
+template <int NW>
+__device__ inline double consumer_sum_double(double v, double* s_dbl, int warp, int lane)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) s_dbl[warp] = v;
+    asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+    double tot = 0.0;
+    if (warp == 0 && lane == 0)
+        for (int w = 0; w < NW; ++w) tot += s_dbl[w];
+    return tot;
+}
+
+// Called by consumer thread 0 of every block when the block has finished its rows: publishes the
+// block's two partial sums; the last block to arrive adds all of them in index order and writes the
+// two losses.
+__device__ inline void publish_block_losses(const RowArgs& p, long long N, double sum_pg, double sum_vf)
+{
+    p.partials[2 * blockIdx.x] = sum_pg;
+    p.partials[2 * blockIdx.x + 1] = sum_vf;
+    __threadfence();
+    const unsigned prev = atomicAdd(p.ticket, 1u);
+    if (prev == gridDim.x - 1) {
         __threadfence();
         double a = 0.0, c = 0.0;
         for (unsigned k = 0; k < gridDim.x; ++k) {
