@@ -112,7 +112,7 @@ def visible_gpu_index(local_rank: int) -> int:
 class Path:
     """All buffers of one step, resident on the device, and the step itself (C-ABI calls only)."""
 
-    def __init__(self, w, batch, dev):
+    def __init__(self, w, batch, dev, fused=True):
         import torch
         from paper_2410_15651_b200 import binding
         self.b, self.w, self.binding = batch, w, binding
@@ -120,26 +120,39 @@ class Path:
         self.ws = binding.workspace(B, T, dev)
         f = lambda: torch.empty((B, T), dtype=torch.float32, device=dev)
         self.lp_act, self.lp_ref, self.rewards, self.adv, self.ret = f(), f(), f(), f(), f()
+        self.exp = binding.Experience(B, T, dev)
+        self.exp.lp_actor, self.exp.lp_ref, self.exp.rewards = self.lp_act, self.lp_ref, self.rewards
+        self.exp.adv, self.exp.returns = self.adv, self.ret
+        self.fused = fused
         self.out = binding.PPOOutputs(batch["actor"])
         self.N = int(batch["lengths"].sum().item())
         # old-policy log-probs = current + N(0, sigma^2) on valid tokens, prepared once outside the timed region
         cur = binding.gather_logprobs(batch["actor"], batch["ids"], batch["lengths"], self.ws)
         mask = torch.arange(T, device=dev)[None, :] < batch["lengths"][:, None]
         self.lp_old = (cur + batch["lp_old_noise"] * mask).contiguous()
-        self.launches_per_step = 6
+        self.launches_per_step = 3 if fused else 5      # kernels of this library per step
 
     def step(self, ev=None):
         b, w, k = self.b, self.w, self.binding
-        k.gather_logprobs(b["actor"], b["ids"], b["lengths"], self.ws, self.lp_act)
-        k.gather_logprobs(b["ref"], b["ids"], b["lengths"], self.ws, self.lp_ref)
-        k.kl_reward(self.lp_old, self.lp_ref, b["score"], b["lengths"], w.beta_kl, w.reward_clip, self.rewards)
-        k.gae(self.rewards, b["values_old"], b["lengths"], w.gamma, w.lam, self.adv, self.ret)
+        if self.fused:
+            # experience phase in one launch; the KL term uses the old-policy log-probs of the workload
+            k.experience(b["actor"], b["ref"], b["ids"], b["lengths"], b["score"], b["values_old"], w.beta_kl,
+                         w.reward_clip, w.gamma, w.lam, self.ws, self.exp, lp_old=self.lp_old)
+        else:
+            self._experience_separate()
         if ev is not None:
             ev[0].record()
         k.ppo_loss_fwd_bwd(b["actor"], b["ids"], b["lengths"], self.lp_old, self.adv, b["values_new"],
                            b["values_old"], self.ret, w.clip_eps, w.value_clip, float(self.N), self.ws, self.out)
         if ev is not None:
             ev[1].record()
+
+    def _experience_separate(self):
+        b, w, k = self.b, self.w, self.binding
+        k.gather_logprobs(b["actor"], b["ids"], b["lengths"], self.ws, self.lp_act)
+        k.gather_logprobs(b["ref"], b["ids"], b["lengths"], self.ws, self.lp_ref)
+        k.kl_reward(self.lp_old, self.lp_ref, b["score"], b["lengths"], w.beta_kl, w.reward_clip, self.rewards)
+        k.gae(self.rewards, b["values_old"], b["lengths"], w.gamma, w.lam, self.adv, self.ret)
 
 
 def run_ours(args):
@@ -162,7 +175,7 @@ def run_ours(args):
     binding.lib()                                              # fail here, loudly, if not built
     w = inputs.scaled(inputs.WORKLOADS[args.workload], seed=inputs.WORKLOADS[args.workload].seed + 1000 * rank)
     batch = inputs.make_batch(w, device=dev)
-    path = Path(w, batch, dev)
+    path = Path(w, batch, dev, fused=not args.separate_calls)
     B, T, V = w.B, w.T, w.V
     n_valid = path.N
 
@@ -252,11 +265,13 @@ def run_ours(args):
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{args.workload}: B={B} T={T} V={V} bf16 logits, {n_valid} response tokens per GPU",
                    "l2": "inputs larger than L2 (%.2f GB touched per step)" % (step_bytes / 1e9 + 0.0),
-                   "multi_gpu": "independent batch per rank, no data-path collective"},
+                   "multi_gpu": "independent batch per rank, no data-path collective",
+                   "calls_per_step": ("rlhf_gather_logprobs x2, rlhf_kl_reward, rlhf_gae, rlhf_ppo_loss_fwd_bwd"
+                                      if args.separate_calls else "rlhf_experience, rlhf_ppo_loss_fwd_bwd")},
         "clocks": clocks, "gpu_launches": path.launches_per_step * K,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e_steps},
-        "roofline": {"bound": "hbm", "kernel": "rlhf_ppo_loss_fwd_bwd (row kernel + finalisation)",
+        "roofline": {"bound": "hbm", "kernel": "rlhf_ppo_loss_fwd_bwd (one launch: row kernel with fused finalisation)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": peak_src, "traffic": traffic, "ms_per_launch": loss_ms,
                      "algorithmic_bytes_per_launch": loss_bytes,
@@ -364,6 +379,8 @@ def main():
     ap.add_argument("--workload", default="opt", choices=["tiny", "opt", "llama2", "large_vocab", "ragged"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-calls", action="store_true",
+                    help="experience phase as four calls (2 x gather_logprobs, kl_reward, gae) instead of rlhf_experience")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

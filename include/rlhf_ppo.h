@@ -12,6 +12,7 @@
  *   rlhf_kl_reward          per-token reward: KL penalty against the reference + sequence score
  *   rlhf_gae                advantages and returns from rewards and critic values
  *   rlhf_ppo_loss_fwd_bwd   clipped policy and value loss, gradient w.r.t. the logits and values
+ *   rlhf_experience         the first three together (both log-prob passes in one kernel, reward + GAE in another)
  *
  * The paper gives these quantities in prose only; the formulas are the standard definitions and
  * are written out beside each function.
@@ -74,7 +75,7 @@ const char* rlhf_status_string(int status);
 /* Text of the last CUDA runtime error this library saw on the calling thread ("" if none). */
 const char* rlhf_last_cuda_error(void);
 
-/* Bytes of scratch that rlhf_gather_logprobs and rlhf_ppo_loss_fwd_bwd need for a batch of B x T
+/* Bytes of scratch that rlhf_gather_logprobs, rlhf_experience and rlhf_ppo_loss_fwd_bwd need for a batch of B x T
  * tokens: O(B*T), never O(B*T*V) -- at most 16*B*T + 65536.  0 if B or T is not positive.
  * The workspace must be 256-byte aligned and must have been cleared once with rlhf_workspace_init
  * before its first use; it can then be reused by any number of calls on the same stream. */
@@ -129,6 +130,32 @@ int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score,
  */
 int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, int B, int T,
              float gamma, float lambda, float* out_adv, float* out_returns, void* stream);
+
+/*
+ * Steps 1-3 together -- the whole experience phase (Section 2.1: the inferences of the actor,
+ * reference, critic and reward models that turn generated responses into experience).  Computes
+ * exactly what
+ *     rlhf_gather_logprobs(actor) , rlhf_gather_logprobs(reference) , rlhf_kl_reward , rlhf_gae
+ * compute when called in that order, with the same arithmetic (results are bit-identical to the four
+ * calls), in two launches instead of four: one kernel streams both logits tensors, one small kernel
+ * does the reward and the GAE scan of each sequence.
+ *   actor_logits, ref_logits   bf16, each with its own strides, same ids / lengths               read
+ *   score, values_old          as in steps 2 and 3                                                read
+ *   lp_old                     fp32 [B,T] or NULL.  The log-probs of the KL term; NULL (the usual
+ *                              case when the experience is being made) = the actor log-probs
+ *                              computed by this call                                              read
+ *   out_lp_actor, out_lp_ref, out_rewards, out_adv, out_returns   fp32 [B,T], distinct buffers    written
+ *   workspace                  as for step 1
+ * Scalars as in steps 2 and 3.  If the rows of either tensor are not 16-byte aligned the four
+ * separate kernels are launched instead.
+ */
+int rlhf_experience(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
+                    const void* ref_logits, long long ref_stride_b, long long ref_stride_t,
+                    const long long* ids, long long ids_stride_b, const int* lengths,
+                    const float* score, const float* values_old, const float* lp_old,
+                    int B, int T, int V, float beta_kl, float reward_clip, float gamma, float lambda,
+                    float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
+                    float* out_returns, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Step 4 -- clipped PPO losses and their gradients (Section 2.1: the actor is trained to maximise

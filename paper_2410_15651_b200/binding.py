@@ -31,6 +31,8 @@ SIGNATURES = {
     "rlhf_gather_logprobs": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
     "rlhf_kl_reward": (_int, [_vp, _vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
     "rlhf_gae": (_int, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp, _vp]),
+    "rlhf_experience": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp,
+                               _int, _int, _int, _f32, _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "rlhf_ppo_loss_fwd_bwd": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
                                      _int, _int, _int, _f32, _f32, _f32, _vp, _vp,
                                      _vp, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
@@ -181,6 +183,42 @@ def gae(rewards: torch.Tensor, values_old: torch.Tensor, lengths: torch.Tensor, 
     _check(lib().rlhf_gae(rewards.data_ptr(), values_old.data_ptr(), lengths.data_ptr(), B, T, gamma, lam,
                           out_adv.data_ptr(), out_returns.data_ptr(), _stream(rewards)), "rlhf_gae")
     return out_adv, out_returns
+
+
+class Experience:
+    """Buffers written by experience(); reusable from call to call."""
+
+    def __init__(self, B: int, T: int, device):
+        f = lambda: torch.empty((B, T), dtype=torch.float32, device=device)
+        self.lp_actor, self.lp_ref, self.rewards, self.adv, self.returns = f(), f(), f(), f(), f()
+
+
+def experience(actor_logits: torch.Tensor, ref_logits: torch.Tensor, ids: torch.Tensor, lengths: torch.Tensor,
+               score: torch.Tensor, values_old: torch.Tensor, beta_kl: float, reward_clip: float,
+               gamma: float, lam: float, ws: torch.Tensor, out: Optional[Experience] = None,
+               lp_old: Optional[torch.Tensor] = None) -> Experience:
+    B, T, V, asb, ast = _logits(actor_logits, "actor_logits")
+    rB, rT, rV, rsb, rst = _logits(ref_logits, "ref_logits")
+    if (rB, rT, rV) != (B, T, V):
+        raise ValueError("actor and reference logits must have the same shape")
+    isb = _ids(ids, B, T)
+    _lengths(lengths, B)
+    _dev(score, torch.float32, "score")
+    if tuple(score.shape) != (B,) or not score.is_contiguous():
+        raise ValueError("score must be a contiguous [B] tensor")
+    _bt(values_old, B, T, "values_old")
+    if out is None:
+        out = Experience(B, T, actor_logits.device)
+    for name in ("lp_actor", "lp_ref", "rewards", "adv", "returns"):
+        _bt(getattr(out, name), B, T, "out." + name)
+    lp_old_ptr = _bt(lp_old, B, T, "lp_old").data_ptr() if lp_old is not None else None
+    _check(lib().rlhf_experience(
+        actor_logits.data_ptr(), asb, ast, ref_logits.data_ptr(), rsb, rst, ids.data_ptr(), isb,
+        lengths.data_ptr(), score.data_ptr(), values_old.data_ptr(), lp_old_ptr, B, T, V,
+        beta_kl, reward_clip, gamma, lam, out.lp_actor.data_ptr(), out.lp_ref.data_ptr(),
+        out.rewards.data_ptr(), out.adv.data_ptr(), out.returns.data_ptr(),
+        ws.data_ptr(), ws.numel(), _stream(actor_logits)), "rlhf_experience")
+    return out
 
 
 class PPOOutputs:

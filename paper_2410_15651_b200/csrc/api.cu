@@ -50,11 +50,14 @@ int check_shape(int B, int T, int V)
     return RLHF_OK;
 }
 
-int check_workspace(const void* ws, size_t bytes, int B, int T)
+// Bytes of the workspace that rlhf_ppo_loss_fwd_bwd touches: header + per-token policy loss terms.
+size_t loss_workspace_bytes(int B, int T) { return kRowLossOffset + 4 * (size_t)B * (size_t)T; }
+
+int check_workspace(const void* ws, size_t bytes, size_t need)
 {
     if (!ws) return RLHF_ERR_NULL;
     if (!aligned(ws, 256)) return RLHF_ERR_ALIGN;
-    if (bytes < rlhf_workspace_bytes(B, T)) return RLHF_ERR_WORKSPACE;
+    if (bytes < need) return RLHF_ERR_WORKSPACE;
     return RLHF_OK;
 }
 
@@ -93,17 +96,17 @@ int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_
 
 constexpr int kLogprobWarps = 24;
 
-int launch_warp_logprob(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
+template <bool kDual>
+int launch_warp_logprob(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream_t s)
 {
-    WarpArgs wa{};
-    wa.row = a;
-    wa.row_bytes = 2u * (unsigned)a.V;
+    WarpArgs wa = wa_in;
+    wa.row_bytes = 2u * (unsigned)wa.row.V;
     const size_t smem = warp_kernel_smem_bytes(kLogprobWarps);
-    const long long rows = (long long)a.B * a.T;
+    const long long rows = (long long)wa.row.B * wa.row.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)smem));
-    logprob_warp_kernel<kLogprobWarps><<<grid, kLogprobWarps * 32, smem, s>>>(wa);
+    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps, kDual>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    logprob_warp_kernel<kLogprobWarps, kDual><<<grid, kLogprobWarps * 32, smem, s>>>(wa);
     return RLHF_OK;
 }
 
@@ -216,7 +219,7 @@ const char* rlhf_last_cuda_error(void) { return g_cuda_error; }
 size_t rlhf_workspace_bytes(int B, int T)
 {
     if (B <= 0 || T <= 0) return 0;
-    size_t n = kRowLossOffset + 4 * (size_t)B * (size_t)T;
+    size_t n = loss_workspace_bytes(B, T);
     return (n + 255) & ~(size_t)255;
 }
 
@@ -254,7 +257,7 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
     if (T > 1 && stride_t < V) return RLHF_ERR_STRIDE;
     if (!aligned(logits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) || !aligned(out_logprobs, 4))
         return RLHF_ERR_ALIGN;
-    if (int e = check_workspace(workspace, workspace_bytes, B, T)) return e;
+    if (int e = check_workspace(workspace, workspace_bytes, rlhf_workspace_bytes(B, T))) return e;
     DeviceInfo dev;
     if (int e = device_info(dev)) return e;
 
@@ -270,7 +273,9 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
     a.out_lp = out_logprobs;
 
     if (rows_16B(logits, stride_b, stride_t, V)) {
-        if (int e = launch_warp_logprob(a, dev, (cudaStream_t)stream)) return e;
+        WarpArgs wa{};
+        wa.row = a;
+        if (int e = launch_warp_logprob<false>(wa, dev, (cudaStream_t)stream)) return e;
         return launch_check("logprob_warp_kernel");
     }
     long long rows = (long long)B * T;
@@ -316,6 +321,77 @@ int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, 
     return launch_check("gae_kernel");
 }
 
+int rlhf_experience(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
+                    const void* ref_logits, long long ref_stride_b, long long ref_stride_t,
+                    const long long* ids, long long ids_stride_b, const int* lengths,
+                    const float* score, const float* values_old, const float* lp_old,
+                    int B, int T, int V, float beta_kl, float reward_clip, float gamma, float lambda,
+                    float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
+                    float* out_returns, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!actor_logits || !ref_logits || !ids || !lengths || !score || !values_old || !out_lp_actor ||
+        !out_lp_ref || !out_rewards || !out_adv || !out_returns)
+        return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, V)) return e;
+    if (actor_stride_b < 0 || actor_stride_t < 0 || ref_stride_b < 0 || ref_stride_t < 0 || ids_stride_b < 0)
+        return RLHF_ERR_STRIDE;
+    if (T > 1 && (actor_stride_t < V || ref_stride_t < V)) return RLHF_ERR_STRIDE;
+    if (!std::isfinite(beta_kl) || beta_kl < 0.f || !std::isfinite(reward_clip) || reward_clip < 0.f ||
+        !(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f))
+        return RLHF_ERR_SCALAR;
+    if (!aligned(actor_logits, 2) || !aligned(ref_logits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) ||
+        !aligned(score, 4) || !aligned(values_old, 4) || (lp_old && !aligned(lp_old, 4)) ||
+        !aligned(out_lp_actor, 4) || !aligned(out_lp_ref, 4) || !aligned(out_rewards, 4) ||
+        !aligned(out_adv, 4) || !aligned(out_returns, 4))
+        return RLHF_ERR_ALIGN;
+    {
+        const float* outs[5] = {out_lp_actor, out_lp_ref, out_rewards, out_adv, out_returns};
+        for (int i = 0; i < 5; ++i) {
+            if (outs[i] == values_old || outs[i] == lp_old) return RLHF_ERR_STRIDE;
+            for (int j = i + 1; j < 5; ++j)
+                if (outs[i] == outs[j]) return RLHF_ERR_STRIDE;
+        }
+    }
+    if (int e = check_workspace(workspace, workspace_bytes, rlhf_workspace_bytes(B, T))) return e;
+
+    if (!rows_16B(actor_logits, actor_stride_b, actor_stride_t, V) ||
+        !rows_16B(ref_logits, ref_stride_b, ref_stride_t, V)) {
+        // unaligned rows: the four steps one after the other
+        if (int e = rlhf_gather_logprobs(actor_logits, actor_stride_b, actor_stride_t, ids, ids_stride_b, lengths,
+                                         B, T, V, out_lp_actor, workspace, workspace_bytes, stream)) return e;
+        if (int e = rlhf_gather_logprobs(ref_logits, ref_stride_b, ref_stride_t, ids, ids_stride_b, lengths,
+                                         B, T, V, out_lp_ref, workspace, workspace_bytes, stream)) return e;
+        if (int e = rlhf_kl_reward(lp_old ? lp_old : out_lp_actor, out_lp_ref, score, lengths, B, T, beta_kl,
+                                   reward_clip, out_rewards, stream)) return e;
+        return rlhf_gae(out_rewards, values_old, lengths, B, T, gamma, lambda, out_adv, out_returns, stream);
+    }
+    DeviceInfo dev;
+    if (int e = device_info(dev)) return e;
+    WarpArgs wa{};
+    wa.row.logits = (const uint16_t*)actor_logits;
+    wa.row.stride_b = actor_stride_b;
+    wa.row.stride_t = actor_stride_t;
+    wa.row.ids = ids;
+    wa.row.ids_stride_b = ids_stride_b;
+    wa.row.lengths = lengths;
+    wa.row.B = B; wa.row.T = T; wa.row.V = V;
+    wa.row.status = (unsigned*)workspace;
+    wa.row.out_lp = out_lp_actor;
+    wa.logits2 = (const uint16_t*)ref_logits;
+    wa.stride2_b = ref_stride_b;
+    wa.stride2_t = ref_stride_t;
+    wa.out_lp2 = out_lp_ref;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (int e = launch_warp_logprob<true>(wa, dev, s)) return e;
+    if (int e = launch_check("logprob_warp_kernel<dual>")) return e;
+    if (int e = keep_max_carveout(reward_gae_kernel)) return e;
+    const int grid = (B + kGaeWarpsPerBlock - 1) / kGaeWarpsPerBlock;
+    reward_gae_kernel<<<grid, kGaeWarpsPerBlock * 32, 0, s>>>(lp_old ? lp_old : out_lp_actor, out_lp_ref, score,
+                                                             values_old, lengths, B, T, beta_kl, reward_clip,
+                                                             gamma, lambda, out_rewards, out_adv, out_returns);
+    return launch_check("reward_gae_kernel");
+}
+
 int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stride_t,
                           const long long* ids, long long ids_stride_b, const int* lengths,
                           const float* lp_old, const float* adv, const float* values_new,
@@ -343,7 +419,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
         !aligned(returns, 4) || !aligned(out_loss_pg, 4) || !aligned(out_loss_vf, 4) ||
         !aligned(out_dvalues, 4) || (out_lp_new && !aligned(out_lp_new, 4)))
         return RLHF_ERR_ALIGN;
-    if (int e = check_workspace(workspace, workspace_bytes, B, T)) return e;
+    if (int e = check_workspace(workspace, workspace_bytes, loss_workspace_bytes(B, T))) return e;
     DeviceInfo dev;
     if (int e = device_info(dev)) return e;
 

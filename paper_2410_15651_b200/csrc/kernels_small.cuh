@@ -7,6 +7,15 @@
 namespace rlhf {
 
 // ---------------------------------------------------------------- step 2: per-token reward
+// r = -beta * (lp_old - lp_ref), plus the clipped sequence score at the last valid token (t == len-1).
+__device__ __forceinline__ float reward_token(float lp_old, float lp_ref, float score, int t, int len,
+                                              float beta, float clip)
+{
+    float r = -beta * (lp_old - lp_ref);
+    if (t == len - 1) r += fminf(fmaxf(score, -clip), clip);
+    return r;
+}
+
 __global__ void __launch_bounds__(256) kl_reward_kernel(const float* __restrict__ lp_old,
                                                         const float* __restrict__ lp_ref,
                                                         const float* __restrict__ score,
@@ -19,10 +28,7 @@ __global__ void __launch_bounds__(256) kl_reward_kernel(const float* __restrict_
         int b = (int)(i / T), t = (int)(i % T);
         int len = clamp_len(__ldg(lengths + b), T);
         float r = 0.f;
-        if (t < len) {
-            r = -beta * (lp_old[i] - lp_ref[i]);
-            if (t == len - 1) r += fminf(fmaxf(__ldg(score + b), -clip), clip);
-        }
+        if (t < len) r = reward_token(lp_old[i], lp_ref[i], __ldg(score + b), t, len, beta, clip);
         out[i] = r;
     }
 }
@@ -34,23 +40,11 @@ __global__ void __launch_bounds__(256) kl_reward_kernel(const float* __restrict_
 // now-known incoming value.  delta_t = r_t + gamma V_{t+1} - V_t with V_len = 0.
 constexpr int kGaeWarpsPerBlock = 4;
 
-__global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) gae_kernel(const float* __restrict__ rewards,
-                                                                     const float* __restrict__ values,
-                                                                     const int* __restrict__ lengths,
-                                                                     int B, int T, float gamma, float lambda,
-                                                                     float* __restrict__ adv,
-                                                                     float* __restrict__ ret)
+// GAE of one sequence by one warp: r, v, a_out, g_out point at the sequence's T entries, n valid.
+__device__ __forceinline__ void gae_warp(const float* r, const float* v, int n, int T, float gamma, float lambda,
+                                         float* a_out, float* g_out, int lane)
 {
-    const int lane = threadIdx.x & 31;
-    const int b = blockIdx.x * kGaeWarpsPerBlock + (threadIdx.x >> 5);
-    if (b >= B) return;
-    const int n = clamp_len(__ldg(lengths + b), T);
-    const float* r = rewards + (long long)b * T;
-    const float* v = values + (long long)b * T;
-    float* a_out = adv + (long long)b * T;
-    float* g_out = ret + (long long)b * T;
     const float q = gamma * lambda;
-
     const int chunk = (n + 31) / 32;
     const int lo = min(n, lane * chunk), hi = min(n, lo + chunk);
 
@@ -87,6 +81,46 @@ __global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) gae_kernel(const float
         }
     }
     for (int t = n + lane; t < T; t += 32) { a_out[t] = 0.f; g_out[t] = 0.f; }
+}
+
+__global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) gae_kernel(const float* __restrict__ rewards,
+                                                                     const float* __restrict__ values,
+                                                                     const int* __restrict__ lengths,
+                                                                     int B, int T, float gamma, float lambda,
+                                                                     float* __restrict__ adv,
+                                                                     float* __restrict__ ret)
+{
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kGaeWarpsPerBlock + (threadIdx.x >> 5);
+    if (b >= B) return;
+    const int n = clamp_len(__ldg(lengths + b), T);
+    gae_warp(rewards + (long long)b * T, values + (long long)b * T, n, T, gamma, lambda,
+             adv + (long long)b * T, ret + (long long)b * T, lane);
+}
+
+// ---------------------------------------------------------------- steps 2+3 in one launch
+// One warp per sequence: the rewards are written first (same formula as kl_reward_kernel), then the
+// warp runs the GAE scan over what it has just written.  Results are bit-identical to the two kernels.
+__global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) reward_gae_kernel(const float* __restrict__ lp_old,
+                                                                            const float* __restrict__ lp_ref,
+                                                                            const float* __restrict__ score,
+                                                                            const float* __restrict__ values,
+                                                                            const int* __restrict__ lengths,
+                                                                            int B, int T, float beta, float clip,
+                                                                            float gamma, float lambda,
+                                                                            float* rewards, float* __restrict__ adv,
+                                                                            float* __restrict__ ret)
+{
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kGaeWarpsPerBlock + (threadIdx.x >> 5);
+    if (b >= B) return;
+    const int n = clamp_len(__ldg(lengths + b), T);
+    const long long off = (long long)b * T;
+    const float sc = __ldg(score + b);
+    for (int t = lane; t < T; t += 32)
+        rewards[off + t] = t < n ? reward_token(lp_old[off + t], lp_ref[off + t], sc, t, n, beta, clip) : 0.f;
+    __syncwarp();
+    gae_warp(rewards + off, values + off, n, T, gamma, lambda, adv + off, ret + off, lane);
 }
 
 // ---------------------------------------------------------------- step 4: finalisation

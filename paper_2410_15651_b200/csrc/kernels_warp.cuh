@@ -34,8 +34,12 @@ __device__ __forceinline__ bool cursor32_seek(Cursor32& c, int k, const int* __r
 }
 
 struct WarpArgs {
-    RowArgs row;
+    RowArgs row;            // logits / out_lp: the (first) tensor
     unsigned row_bytes;     // 2*V, multiple of 16
+    // kDual: a second logits tensor (the reference model's) read with the same ids in the same launch
+    const uint16_t* logits2;
+    long long stride2_b, stride2_t;
+    float* out_lp2;
 };
 
 inline size_t warp_kernel_smem_bytes(int warps_per_block)
@@ -43,7 +47,7 @@ inline size_t warp_kernel_smem_bytes(int warps_per_block)
     return (size_t)warps_per_block * (kWarpSlots * kWarpChunk + kWarpSlots * 8);
 }
 
-template <int WPB>
+template <int WPB, bool kDual>
 __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -55,7 +59,7 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
     const uint32_t ring_addr = smem_u32(ring);
     const uint32_t bar_addr = smem_u32(smem + (size_t)WPB * (kWarpSlots * kWarpChunk)) + (uint32_t)warp * (kWarpSlots * 8);
 
-    const int N = (int)block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
+    const int N1 = (int)block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
     if (lane == 0) {
         for (int s = 0; s < kWarpSlots; ++s) mbar_init(bar_addr + 8u * s, 1);
         fence_mbar_init();
@@ -67,12 +71,16 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
         const long long total = (long long)p.B * p.T;
         for (long long i = (long long)blockIdx.x * blockDim.x + tid; i < total; i += (long long)gridDim.x * blockDim.x) {
             int b = (int)(i / p.T), t = (int)(i % p.T);
-            if (t >= clamp_len(__ldg(p.lengths + b), p.T)) p.out_lp[i] = 0.f;
+            if (t >= clamp_len(__ldg(p.lengths + b), p.T)) {
+                p.out_lp[i] = 0.f;
+                if (kDual) wa.out_lp2[i] = 0.f;
+            }
         }
     }
 
     // rows are dealt to blocks first, then to warps: consecutive rows go to different SMs, and a batch
     // with fewer rows than warps still loads every SM equally
+    const int N = kDual ? 2 * N1 : N1;                              // rows: tensor 1, then tensor 2
     const int gw = warp * (int)gridDim.x + (int)blockIdx.x;       // this warp's first row
     const int GW = (int)gridDim.x * WPB;
     const uint32_t nvec = wa.row_bytes / 16u;
@@ -85,10 +93,14 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
     int ic = 0;                 // its chunk index
     int islot = 0;
     const unsigned char* irow = nullptr;
+    bool iwrapped = false;
     auto issue_seek = [&]() {
         int b, t;
-        if (ik < N && cursor32_seek(icur, ik, p.lengths, p.B, p.T, b, t))
-            irow = (const unsigned char*)(p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t);
+        const bool second = kDual && ik >= N1;
+        if (second && !iwrapped) { icur = Cursor32{0, 0}; iwrapped = true; }
+        if (ik < N && cursor32_seek(icur, second ? ik - N1 : ik, p.lengths, p.B, p.T, b, t))
+            irow = second ? (const unsigned char*)(wa.logits2 + (long long)b * wa.stride2_b + (long long)t * wa.stride2_t)
+                          : (const unsigned char*)(p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t);
         else
             ik = N;
     };
@@ -113,8 +125,11 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
     uint32_t phases = 0;        // bit s: parity to wait for on slot s
     int nb = 0, nt = 0;
     long long ny = 0;
+    bool wrapped = false;
     auto fetch_row = [&](int k) {
-        if (k < N && cursor32_seek(cur, k, p.lengths, p.B, p.T, nb, nt))
+        const bool second = kDual && k >= N1;
+        if (second && !wrapped) { cur = Cursor32{0, 0}; wrapped = true; }
+        if (k < N && cursor32_seek(cur, second ? k - N1 : k, p.lengths, p.B, p.T, nb, nt))
             ny = __ldg(p.ids + (long long)nb * p.ids_stride_b + nt);
     };
     fetch_row(gw);
@@ -180,7 +195,8 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
         zy = __shfl_sync(0xffffffffu, zy, owner);
         if (lane == 0 && !aborted) {
             const RowResult r = row_finish(Acc{M, s, ey}, zy);
-            p.out_lp[flat] = bad_id ? 0.f : r.lp;
+            float* out = (kDual && k >= N1) ? wa.out_lp2 : p.out_lp;
+            out[flat] = bad_id ? 0.f : r.lp;
         }
     }
 }

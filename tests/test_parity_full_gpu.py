@@ -13,7 +13,7 @@ import torch
 from paper_2410_15651_b200 import binding, inputs
 
 from helpers import OracleRun
-from test_parity_gpu import DEV, dlogits_properties, run_steps, sample_rows
+from test_parity_gpu import DEV, _experience_both_ways, dlogits_properties, run_steps, sample_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -28,6 +28,8 @@ def test_full_size(oracle, name, in_place):
     out, rep = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"],
                          in_place=in_place, sample_rows=rows)
     dlogits_properties(run, out, batch["ids"], batch["actor"])
+    if not in_place:
+        _experience_both_ways(w, batch, batch["actor"], batch["ref"], batch["ids"])
     print(name, {k: (round(v, 4) if isinstance(v, float) else v) for k, v in rep.items()})
     del batch, out
     torch.cuda.empty_cache()

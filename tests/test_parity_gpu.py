@@ -222,3 +222,65 @@ def test_gae_long_sequences_closed_form(oracle):
         adv, ret = binding.gae(_t(r), _t(v), _t(lengths, torch.int32), gamma, lam)
         wa, wr = oracle.gae(r, v, lengths, gamma, lam)
         assert close_rel(np32(adv), wa)[0] and close_rel(np32(ret), wr)[0]
+
+
+def _experience_both_ways(w, batch, logits, ref, ids, lp_old=None):
+    """rlhf_experience against the four separate calls it stands for: bit-identical outputs."""
+    B, T, _ = logits.shape
+    lengths = batch["lengths"]
+    ws = binding.workspace(B, T, DEV)
+    lp_a = binding.gather_logprobs(logits, ids, lengths, ws)
+    lp_r = binding.gather_logprobs(ref, ids, lengths, ws)
+    r = binding.kl_reward(lp_a if lp_old is None else lp_old, lp_r, batch["score"], lengths, w.beta_kl, w.reward_clip)
+    adv, ret = binding.gae(r, batch["values_old"], lengths, w.gamma, w.lam)
+    out = binding.Experience(B, T, DEV)
+    for t in (out.lp_actor, out.lp_ref, out.rewards, out.adv, out.returns):
+        t.fill_(float("nan"))
+    for _ in range(2):                       # twice: the per-sequence counters in the workspace must come back to zero
+        binding.experience(logits, ref, ids, lengths, batch["score"], batch["values_old"], w.beta_kl,
+                           w.reward_clip, w.gamma, w.lam, ws, out, lp_old=lp_old)
+        assert binding.poll_status(ws) == 0
+        for name, got, want in (("lp_actor", out.lp_actor, lp_a), ("lp_ref", out.lp_ref, lp_r),
+                                ("rewards", out.rewards, r), ("adv", out.adv, adv), ("returns", out.returns, ret)):
+            assert torch.equal(got, want), name
+    return out
+
+
+def test_experience_fused_tiny_and_ragged(oracle):
+    w = inputs.WORKLOADS["tiny"]
+    batch = inputs.make_batch(w, device=DEV)
+    out = _experience_both_ways(w, batch, batch["actor"], batch["ref"], batch["ids"])
+    # and against the oracle, the KL term taken from the actor log-probs computed in the same call
+    ln = batch["lengths"].cpu().numpy()
+    from helpers import bits
+    o_a = oracle.gather_logprobs(bits(batch["actor"]), batch["ids"].cpu().numpy(), ln)
+    o_r = oracle.gather_logprobs(bits(batch["ref"]), batch["ids"].cpu().numpy(), ln)
+    o_rw = oracle.kl_reward(np32(out.lp_actor), np32(out.lp_ref), np32(batch["score"]), ln, w.beta_kl, w.reward_clip)
+    o_adv, o_ret = oracle.gae(np32(out.rewards), np32(batch["values_old"]), ln, w.gamma, w.lam)
+    assert np.abs(np32(out.lp_actor) - o_a).max() <= TOL_LP and np.abs(np32(out.lp_ref) - o_r).max() <= TOL_LP
+    assert close_rel(np32(out.rewards), o_rw)[0] and close_rel(np32(out.adv), o_adv)[0] and close_rel(np32(out.returns), o_ret)[0]
+    # ragged recipe: empty sequences, lengths 1 and 2, -inf entries; with an explicit lp_old for the KL term
+    w2 = inputs.scaled(inputs.WORKLOADS["ragged"], B=12, T=40, V=4096)
+    b2 = inputs.make_batch(w2, device=DEV)
+    _experience_both_ways(w2, b2, b2["actor"], b2["ref"], b2["ids"])
+    lp_old = torch.randn((12, 40), device=DEV) - 5.0
+    _experience_both_ways(w2, b2, b2["actor"], b2["ref"], b2["ids"], lp_old=lp_old)
+    # all padding
+    w3 = inputs.scaled(w, lengths="uniform:0:0")
+    b3 = inputs.make_batch(w3, device=DEV)
+    o3 = _experience_both_ways(w3, b3, b3["actor"], b3["ref"], b3["ids"])
+    assert (o3.rewards == 0).all() and (o3.adv == 0).all() and (o3.returns == 0).all()
+
+
+@pytest.mark.parametrize("V", [1001, 7])
+def test_experience_unaligned_rows_take_the_separate_kernels(V):
+    w = inputs.scaled(inputs.WORKLOADS["tiny"], V=V, B=3, T=9, lengths="uniform:0:9", seed=40 + V)
+    batch = inputs.make_batch(w, device=DEV)
+    _experience_both_ways(w, batch, batch["actor"], batch["ref"], batch["ids"])
+
+
+def test_experience_strided_views():
+    w = inputs.WORKLOADS["tiny"]
+    full = inputs.make_batch(w, device=DEV, with_prompt=True)
+    _experience_both_ways(w, full, inputs.response_view(w, full["actor"]), inputs.response_view(w, full["ref"]),
+                          full["ids"][:, w.P:])
