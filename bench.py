@@ -158,7 +158,7 @@ class Path:
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2410_15651_b200 import binding, inputs
+    from paper_2410_15651_b200 import binding, inputs, parallel
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -206,15 +206,10 @@ def run_ours(args):
     loss_ms = sum(a.elapsed_time(b) for a, b in inner) / K
     assert binding.poll_status(path.ws) == 0
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-        n = torch.tensor([n_valid], device=dev, dtype=torch.float64)
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-        total_tokens = float(n.item())
-    else:
-        total_tokens = float(n_valid)
+    # whole-job numbers: the slowest rank's time, the tokens of all ranks
+    elapsed_ms = parallel.max_over_ranks(elapsed_ms, dev)
+    loss_ms = parallel.max_over_ranks(loss_ms, dev)
+    total_tokens = parallel.sum_over_ranks(float(n_valid), dev)
     ms_per_step = elapsed_ms / K
     value = total_tokens / (ms_per_step * 1e-3)
 
@@ -244,10 +239,7 @@ def run_ours(args):
     e1.record()
     sync_all()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = parallel.max_over_ranks(e2e_ms, dev)
     e2e_value = total_tokens / (e2e_ms / e_steps * 1e-3)
 
     # ---- roofline of the dominant kernel (the loss forward/backward)
