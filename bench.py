@@ -174,6 +174,8 @@ def run_ours(args):
 
     binding.lib()                                              # fail here, loudly, if not built
     w = inputs.scaled(inputs.WORKLOADS[args.workload], seed=inputs.WORKLOADS[args.workload].seed + 1000 * rank)
+    if args.sequences > 0:
+        w = inputs.scaled(w, B=args.sequences)
     batch = inputs.make_batch(w, device=dev)
     path = Path(w, batch, dev, fused=not args.separate_calls)
     B, T, V = w.B, w.T, w.V
@@ -370,6 +372,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="opt", choices=["tiny", "opt", "llama2", "large_vocab", "ragged"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sequences", type=int, default=0,
+                    help="override the number of sequences B of the workload (smaller cases for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-calls", action="store_true",
                     help="experience phase as four calls (2 x gather_logprobs, kl_reward, gae) instead of rlhf_experience")
