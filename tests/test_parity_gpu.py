@@ -284,3 +284,22 @@ def test_experience_strided_views():
     full = inputs.make_batch(w, device=DEV, with_prompt=True)
     _experience_both_ways(w, full, inputs.response_view(w, full["actor"]), inputs.response_view(w, full["ref"]),
                           full["ids"][:, w.P:])
+
+
+@pytest.mark.parametrize("V,in_place", [(65544, False), (70000, True), (131072, False), (57000, False)])
+def test_rows_larger_than_shared_memory(oracle, V, in_place):
+    # rows above 111 KB are cut into 64 KB tiles and streamed twice: two tiles plus 16 bytes, a ragged last
+    # tile, exactly four tiles; 57000 (114,000 B) is the first size past the two-resident-rows kernel
+    w = inputs.scaled(inputs.WORKLOADS["ragged"], V=V, B=5, T=6, seed=70 + V % 7)
+    batch = inputs.make_batch(w, device=DEV)
+    batch["lengths"] = torch.tensor([0, 1, 6, 3, 6], dtype=torch.int32, device=DEV)
+    # labels in the first, the last and a middle vector of the row
+    batch["ids"][2, 0], batch["ids"][2, 1], batch["ids"][2, 2] = 0, V - 1, V // 2
+    batch["actor"][2, 1, V - 1] = 3.0
+    batch["actor"][2, 2, V // 2] = 2.0
+    batch["actor"][2, 0, 0] = 1.0
+    batch["ref"][2, :3] = batch["actor"][2, :3]
+    run = OracleRun(oracle, w, batch)
+    out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], in_place=in_place, all_rows=True)
+    if not in_place:
+        dlogits_properties(run, out, batch["ids"], batch["actor"])
