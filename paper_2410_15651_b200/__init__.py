@@ -5,4 +5,4 @@
 synthetic workloads.  Importing the package loads nothing; the library is loaded on first use
 and the call fails loudly if it has not been built.
 """
-__all__ = ["binding", "inputs", "build", "parallel"]
+__all__ = ["binding", "inputs", "build", "parallel", "memory"]
