@@ -370,7 +370,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="opt", choices=["tiny", "opt", "llama2", "large_vocab", "ragged"])
+    ap.add_argument("--workload", default="opt", choices=["tiny", "opt", "llama2", "large_vocab", "ragged", "gpt2"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sequences", type=int, default=0,
                     help="override the number of sequences B of the workload (smaller cases for profiling)")

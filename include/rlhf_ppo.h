@@ -146,8 +146,7 @@ int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, 
  *                              computed by this call                                              read
  *   out_lp_actor, out_lp_ref, out_rewards, out_adv, out_returns   fp32 [B,T], distinct buffers    written
  *   workspace                  as for step 1
- * Scalars as in steps 2 and 3.  If the rows of either tensor are not 16-byte aligned the four
- * separate kernels are launched instead.
+ * Scalars as in steps 2 and 3.
  */
 int rlhf_experience(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
                     const void* ref_logits, long long ref_stride_b, long long ref_stride_t,

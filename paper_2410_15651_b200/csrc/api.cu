@@ -96,7 +96,7 @@ int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_
 
 constexpr int kLogprobWarps = 24;
 
-template <bool kDual>
+template <bool kDual, bool kAny = false>
 int launch_warp_logprob(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream_t s)
 {
     WarpArgs wa = wa_in;
@@ -104,9 +104,9 @@ int launch_warp_logprob(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream
     const size_t smem = warp_kernel_smem_bytes(kLogprobWarps);
     const long long rows = (long long)wa.row.B * wa.row.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps, kDual>,
+    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps, kDual, kAny>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    logprob_warp_kernel<kLogprobWarps, kDual><<<grid, kLogprobWarps * 32, smem, s>>>(wa);
+    logprob_warp_kernel<kLogprobWarps, kDual, kAny><<<grid, kLogprobWarps * 32, smem, s>>>(wa);
     return RLHF_OK;
 }
 
@@ -272,16 +272,15 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
     a.status = (unsigned*)workspace;
     a.out_lp = out_logprobs;
 
+    WarpArgs wa{};
+    wa.row = a;
     if (rows_16B(logits, stride_b, stride_t, V)) {
-        WarpArgs wa{};
-        wa.row = a;
-        if (int e = launch_warp_logprob<false>(wa, dev, (cudaStream_t)stream)) return e;
-        return launch_check("logprob_warp_kernel");
+        if (int e = launch_warp_logprob<false, false>(wa, dev, (cudaStream_t)stream)) return e;
+    } else {
+        // rows that start or end off a 16-byte boundary (odd V, odd strides): same kernel, aligned spans
+        if (int e = launch_warp_logprob<false, true>(wa, dev, (cudaStream_t)stream)) return e;
     }
-    long long rows = (long long)B * T;
-    int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
-    row_generic_kernel<false><<<grid, kGenericThreads, 0, (cudaStream_t)stream>>>(a);
-    return launch_check("row_generic_kernel<logprob>");
+    return launch_check("logprob_warp_kernel");
 }
 
 int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score, const int* lengths,
@@ -354,17 +353,8 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     }
     if (int e = check_workspace(workspace, workspace_bytes, rlhf_workspace_bytes(B, T))) return e;
 
-    if (!rows_16B(actor_logits, actor_stride_b, actor_stride_t, V) ||
-        !rows_16B(ref_logits, ref_stride_b, ref_stride_t, V)) {
-        // unaligned rows: the four steps one after the other
-        if (int e = rlhf_gather_logprobs(actor_logits, actor_stride_b, actor_stride_t, ids, ids_stride_b, lengths,
-                                         B, T, V, out_lp_actor, workspace, workspace_bytes, stream)) return e;
-        if (int e = rlhf_gather_logprobs(ref_logits, ref_stride_b, ref_stride_t, ids, ids_stride_b, lengths,
-                                         B, T, V, out_lp_ref, workspace, workspace_bytes, stream)) return e;
-        if (int e = rlhf_kl_reward(lp_old ? lp_old : out_lp_actor, out_lp_ref, score, lengths, B, T, beta_kl,
-                                   reward_clip, out_rewards, stream)) return e;
-        return rlhf_gae(out_rewards, values_old, lengths, B, T, gamma, lambda, out_adv, out_returns, stream);
-    }
+    const bool all_16B = rows_16B(actor_logits, actor_stride_b, actor_stride_t, V) &&
+                         rows_16B(ref_logits, ref_stride_b, ref_stride_t, V);
     DeviceInfo dev;
     if (int e = device_info(dev)) return e;
     WarpArgs wa{};
@@ -382,7 +372,11 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     wa.stride2_t = ref_stride_t;
     wa.out_lp2 = out_lp_ref;
     cudaStream_t s = (cudaStream_t)stream;
-    if (int e = launch_warp_logprob<true>(wa, dev, s)) return e;
+    if (all_16B) {
+        if (int e = launch_warp_logprob<true, false>(wa, dev, s)) return e;
+    } else {
+        if (int e = launch_warp_logprob<true, true>(wa, dev, s)) return e;
+    }
     if (int e = launch_check("logprob_warp_kernel<dual>")) return e;
     if (int e = keep_max_carveout(reward_gae_kernel)) return e;
     const int grid = (B + kGaeWarpsPerBlock - 1) / kGaeWarpsPerBlock;

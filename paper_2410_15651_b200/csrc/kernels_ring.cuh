@@ -153,6 +153,23 @@ __device__ __forceinline__ float acc_add_vec_label(Acc& a, const uint4& q, int j
     return zy;
 }
 
+// A vector of which only entries jlo <= j < jhi belong to the row (the first or last vector of a row that
+// does not start or end on a 16-byte boundary); entry jlabel, if in range, is the generated token.
+__device__ __forceinline__ float acc_add_vec_range(Acc& a, const uint4& q, int jlo, int jhi, int jlabel)
+{
+    float z[8];
+    unpack8(q, z);
+    float zy = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (i >= jlo && i < jhi) {
+            acc_add(a, z[i], i == jlabel);
+            if (i == jlabel) zy = z[i];
+        }
+    }
+    return zy;
+}
+
 // dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.
 __device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sign2)
 {

@@ -47,7 +47,11 @@ inline size_t warp_kernel_smem_bytes(int warps_per_block)
     return (size_t)warps_per_block * (kWarpSlots * kWarpChunk + kWarpSlots * 8);
 }
 
-template <int WPB, bool kDual>
+// kAny: rows may start at any even byte address and have any length (V not a multiple of 8): every row
+// is then loaded as the 16-byte aligned span that contains it, and the entries of the first and last
+// vector that lie outside the row are skipped.  (The span stays inside the 16-byte blocks that hold the
+// row's first and last element.)
+template <int WPB, bool kDual, bool kAny>
 __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -93,6 +97,8 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
     int ic = 0;                 // its chunk index
     int islot = 0;
     const unsigned char* irow = nullptr;
+    uint32_t ispan = wa.row_bytes;    // bytes to load for the row being requested
+    int inchunks = nchunks;
     bool iwrapped = false;
     auto issue_seek = [&]() {
         int b, t;
@@ -103,15 +109,21 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
                           : (const unsigned char*)(p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t);
         else
             ik = N;
+        if (kAny && ik < N) {
+            const uint32_t mis = (uint32_t)((uintptr_t)irow & 15u);
+            irow -= mis;
+            ispan = (mis + wa.row_bytes + 15u) & ~15u;
+            inchunks = (int)((ispan + kWarpChunk - 1) / kWarpChunk);
+        }
     };
     auto issue_next = [&]() {
         if (ik >= N) return;
         const uint32_t off = (uint32_t)ic * kWarpChunk;
-        const uint32_t bytes = min((uint32_t)kWarpChunk, wa.row_bytes - off);
+        const uint32_t bytes = min((uint32_t)kWarpChunk, ispan - off);
         mbar_arrive_expect_tx(bar_addr + 8u * islot, bytes);
         bulk_load(ring_addr + (uint32_t)islot * kWarpChunk, irow + off, bytes, bar_addr + 8u * islot);
         islot = islot + 1 == kWarpSlots ? 0 : islot + 1;
-        if (++ic == nchunks) { ic = 0; ik += GW; issue_seek(); }
+        if (++ic == inchunks) { ic = 0; ik += GW; issue_seek(); }
     };
     if (lane == 0) {
         issue_seek();
@@ -139,18 +151,33 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
         long long y = ny;
         const bool bad_id = (y < 0 || y >= p.V);
         if (bad_id) { y = 0; if (lane == 0) atomicOr(p.status, kErrIdRange); }
-        const uint32_t yvec = (uint32_t)(y >> 3);
-        const int yj = (int)(y & 7);
+        // where the row sits in the loaded span: eoff entries of the first vector precede it
+        uint32_t eoff = 0, row_vecs = nvec;
+        int row_chunks = nchunks, plain_end = full_chunks;         // chunks [plain_begin, plain_end) hold only whole vectors of the row
+        if (kAny) {
+            const bool second = kDual && k >= N1;
+            const uint16_t* rp = second ? wa.logits2 + (long long)nb * wa.stride2_b + (long long)nt * wa.stride2_t
+                                        : p.logits + (long long)nb * p.stride_b + (long long)nt * p.stride_t;
+            const uint32_t mis = (uint32_t)((uintptr_t)rp & 15u);
+            eoff = mis >> 1;
+            const uint32_t span = (mis + wa.row_bytes + 15u) & ~15u;
+            row_vecs = span / 16u;
+            row_chunks = (int)((span + kWarpChunk - 1) / kWarpChunk);
+            plain_end = (int)(((eoff + (uint32_t)p.V) >> 3) / kWarpChunkVecs);
+        }
+        const int plain_begin = (kAny && eoff != 0) ? 1 : 0;
+        const uint32_t yvec = (uint32_t)((eoff + (uint32_t)y) >> 3);
+        const int yj = (int)((eoff + (uint32_t)y) & 7);
         const int ychunk = (int)(yvec / kWarpChunkVecs);
         fetch_row(k + GW);                                          // next row's token id, in flight during this row
 
         Acc a = acc_empty();
         float zy = 0.f;
-        for (int c = 0; c < nchunks; ++c) {
+        for (int c = 0; c < row_chunks; ++c) {
             mbar_wait(bar_addr + 8u * slot, (phases >> slot) & 1u, p.status, aborted);
             phases ^= 1u << slot;
             const uint4* src = (const uint4*)(ring + (size_t)slot * kWarpChunk) + lane;
-            if (c < full_chunks && c != ychunk) {
+            if (c >= plain_begin && c < plain_end && c != ychunk) {
                 if (c == 0) a.M = max8_scaled(src[0]);             // this lane's reference exponent for the row
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -170,9 +197,12 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const uint32_t v = v0 + u * 32;
-                    if (v < nvec) {
+                    if (v < row_vecs) {
                         const uint4 q = src[u * 32];
-                        if (v == yvec) zy = acc_add_vec_label(a, q, yj);
+                        const int e0 = (int)(v * 8u) - (int)eoff;      // row index of the vector's first entry
+                        if (kAny && (e0 < 0 || e0 + 8 > p.V))
+                            zy += acc_add_vec_range(a, q, max(0, -e0), min(8, p.V - e0), v == yvec ? yj : -1);
+                        else if (v == yvec) zy = acc_add_vec_label(a, q, yj);
                         else acc_add_vec(a, q);
                     }
                 }

@@ -59,6 +59,9 @@ WORKLOADS: Dict[str, Workload] = {
                        lengths="uniform:64:512", seed=2),
     "large_vocab": Workload("large_vocab", B=64, T=512, V=128256, logit_sigma=4.0, ref_sigma=0.2,
                             lengths="full", seed=3),
+    # beyond the five configurations: the paper's second model family, GPT-2 (vocabulary 50257: rows are
+    # 100,514 bytes long, so consecutive rows start 2 bytes further off a 16-byte boundary)
+    "gpt2": Workload("gpt2", B=16, P=256, T=256, V=50257, ids="softmax", lengths="uniform:128:256", seed=5),
     "ragged": Workload("ragged", B=128, T=1024, V=50272, lengths="mixture", temp_rows=0.5,
                        temperature=0.3, neg_inf_rows=0.25, neg_inf_frac=0.01,
                        gamma=0.99, lam=1.0, seed=4),

@@ -303,3 +303,21 @@ def test_rows_larger_than_shared_memory(oracle, V, in_place):
     out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], in_place=in_place, all_rows=True)
     if not in_place:
         dlogits_properties(run, out, batch["ids"], batch["actor"])
+
+
+def test_gpt2_vocabulary_rows_off_16_byte_boundaries(oracle):
+    # V = 50257: every row starts 2 bytes further off a 16-byte boundary than the one before it
+    w = inputs.scaled(inputs.WORKLOADS["gpt2"], B=3, T=12, lengths="uniform:5:12")
+    batch = inputs.make_batch(w, device=DEV)
+    batch["ids"][0, 0], batch["ids"][0, 1], batch["ids"][1, 0] = 0, w.V - 1, 7       # labels in the ragged first/last vectors
+    batch["actor"][0, 0, 0], batch["actor"][0, 1, w.V - 1], batch["actor"][1, 0, 7] = 4.0, 4.0, 4.0
+    run = OracleRun(oracle, w, batch)
+    out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    _experience_both_ways(w, batch, batch["actor"], batch["ref"], batch["ids"])
+    # a view that starts in the middle of a row of a larger tensor: odd base address as well
+    big = torch.zeros((3, 12, w.V + 5), dtype=torch.bfloat16, device=DEV)
+    big[:, :, 3:3 + w.V] = batch["actor"]
+    view = big[:, :, 3:3 + w.V]
+    ws = binding.workspace(w.B, w.T, DEV)
+    lp = binding.gather_logprobs(view, batch["ids"], batch["lengths"], ws)
+    assert np.abs(np32(lp).astype(np.float64) - run.lp_actor).max() <= TOL_LP
