@@ -113,31 +113,24 @@ int launch_warp_logprob(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream
 constexpr int kDbufWarps = 16;
 
 // Loss kernel for rows of which two fit in shared memory; returns false if the row is out of its range.
-bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev)
+bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev, bool any_alignment = false)
 {
-    return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes) + 1280 <= (size_t)dev.max_smem_optin;
+    return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes, any_alignment) + 1280 <= (size_t)dev.max_smem_optin;
 }
 
-template <int NW>
-int launch_dbuf_as(const DbufArgs& da, size_t smem, int grid, cudaStream_t s)
-{
-    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    loss_dbuf_kernel<NW><<<grid, NW * 32 + 32, smem, s>>>(da);
-    return RLHF_OK;
-}
-
+template <bool kAny>
 int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 {
     DbufArgs da{};
     da.row = a;
     da.row_bytes = 2u * (unsigned)a.V;
-    da.row_stride = (da.row_bytes + 127u) & ~127u;
-    const size_t smem = dbuf_smem_bytes(da.row_bytes);
+    da.row_stride = (unsigned)dbuf_row_stride(da.row_bytes, kAny);
+    const size_t smem = dbuf_smem_bytes(da.row_bytes, kAny);
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    const char* tune = getenv("RLHF_TUNE_DBUF_WARPS");
-    if (tune && atoi(tune) == 24) return launch_dbuf_as<24>(da, smem, grid, s);
-    return launch_dbuf_as<kDbufWarps>(da, smem, grid, s);
+    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps, kAny>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    loss_dbuf_kernel<kDbufWarps, kAny><<<grid, kDbufWarps * 32 + 32, smem, s>>>(da);
+    return RLHF_OK;
 }
 
 template <bool kLoss>
@@ -145,7 +138,7 @@ int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 {
     const unsigned row_bytes = 2u * (unsigned)a.V;
     if constexpr (kLoss) {
-        if (dbuf_applies(row_bytes, dev)) return launch_dbuf(a, dev, s);
+        if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false>(a, dev, s);
     }
     const RingPlan pl = plan_ring(row_bytes, kLoss, dev.smem_per_sm, dev.max_smem_optin);
     RingArgs ra{};
@@ -439,8 +432,13 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
 
     cudaStream_t s = (cudaStream_t)stream;
     long long rows = (long long)B * T;
-    if (rows_16B(logits, stride_b, stride_t, V) && rows_16B(out_dlogits, dl_stride_b, dl_stride_t, V) &&
-        dev.sm_count * 7 <= kMaxFusedBlocks) {
+    const bool all_16B = rows_16B(logits, stride_b, stride_t, V) && rows_16B(out_dlogits, dl_stride_b, dl_stride_t, V);
+    // rows off 16-byte boundaries can still take the two-resident-rows kernel if every dlogits row is as far
+    // off a boundary as its logits row (in place, or a second tensor of the same layout)
+    const bool same_offsets = ((reinterpret_cast<uintptr_t>(out_dlogits) - reinterpret_cast<uintptr_t>(logits)) % 16) == 0 &&
+                              ((dl_stride_b - stride_b) % 8) == 0 && ((dl_stride_t - stride_t) % 8) == 0;
+    const bool ragged_fast = !all_16B && same_offsets && dbuf_applies(2u * (unsigned)V, dev, true);
+    if ((all_16B || ragged_fast) && dev.sm_count * 7 <= kMaxFusedBlocks) {
         // fast path: the row kernel also does the finalisation (value loss, dvalues, loss reduction)
         a.fused = 1;
         a.values_new = values_new;
@@ -452,7 +450,11 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
         a.out_loss_vf = out_loss_vf;
         a.ticket = (unsigned*)(ws + 4);
         a.partials = (double*)(ws + kPartialsOffset);
-        if (int e = launch_ring<true>(a, dev, s)) return e;
+        if (ragged_fast) {
+            if (int e = launch_dbuf<true>(a, dev, s)) return e;
+        } else {
+            if (int e = launch_ring<true>(a, dev, s)) return e;
+        }
         return launch_check("loss row kernel");
     } else {
         int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);

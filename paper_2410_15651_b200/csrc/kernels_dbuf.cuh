@@ -36,11 +36,18 @@ struct RowInfo {
     int bad_id;
     float lp_old;
     float adv;
+    unsigned mis;           // bytes between the 16-byte boundary below the row's first logit and that logit
+    unsigned pad;
 };
 
-inline size_t dbuf_smem_bytes(unsigned row_bytes)
+inline size_t dbuf_row_stride(unsigned row_bytes, bool any_alignment)
 {
-    const size_t stride = ((size_t)row_bytes + 127) & ~(size_t)127;
+    return ((size_t)row_bytes + (any_alignment ? 16 : 0) + 127) & ~(size_t)127;
+}
+
+inline size_t dbuf_smem_bytes(unsigned row_bytes, bool any_alignment = false)
+{
+    const size_t stride = dbuf_row_stride(row_bytes, any_alignment);
     return 2 * stride + kZeroBytes + 64;       // + 6 mbarriers
 }
 
@@ -75,7 +82,11 @@ __device__ __forceinline__ Acc dbuf_reduce(const Acc& a, float2* s_part, const L
     return tot;
 }
 
-template <int NW>
+// kAny: rows (of logits and dlogits alike, with the same offset from a 16-byte boundary) may start at any
+// even address and have any length.  The aligned span around the row is loaded; entries of its first and
+// last vector outside the row are skipped in pass 1 and never stored: the whole vectors inside the row go
+// out by bulk store, the ragged ends by 2-byte stores.
+template <int NW, bool kAny>
 __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
 {
     constexpr int kCons = NW * 32;
@@ -130,8 +141,16 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
             int b, t;
             if (!cursor_seek_padded(pcur, blockIdx.x + pads_done * G, p.lengths, p.B, p.T, b, t)) return;
             unsigned char* drow = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t);
-            for (uint32_t off = 0; off < da.row_bytes; off += kZeroBytes)
-                bulk_store(drow + off, smem_u32(zero_buf), min((uint32_t)kZeroBytes, da.row_bytes - off));
+            uint32_t lo = 0, hi = da.row_bytes;                  // [lo,hi): the part of the row made of whole 16-byte vectors
+            if (kAny) {
+                const uint32_t mis = (uint32_t)((uintptr_t)drow & 15u);
+                lo = min(da.row_bytes, (16u - mis) & 15u);
+                hi = max(lo, da.row_bytes - ((mis + da.row_bytes) & 15u));
+                for (uint32_t o = 0; o < lo; o += 2) *(uint16_t*)(drow + o) = 0;
+                for (uint32_t o = hi; o < da.row_bytes; o += 2) *(uint16_t*)(drow + o) = 0;
+            }
+            for (uint32_t off = lo; off < hi; off += kZeroBytes)
+                bulk_store(drow + off, smem_u32(zero_buf), min((uint32_t)kZeroBytes, hi - off));
             bulk_commit();
         };
         // Hands buffer (i&1), holding the finished gradient of this block's i-th row, to the bulk-store
@@ -142,8 +161,20 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
             mbar_wait(computed(buf), (uint32_t)(i >> 1) & 1u, p.status, aborted);
             if (aborted) return;
             const uint32_t srcb = buf_addr + (uint32_t)buf * da.row_stride;
-            for (uint32_t off = 0; off < da.row_bytes; off += kPiece)
-                bulk_store((buf ? drow1 : drow0) + off, srcb + off, min(kPiece, da.row_bytes - off));
+            unsigned char* drow = buf ? drow1 : drow0;               // the row's first entry in global memory
+            uint32_t mis = 0, lo = 0, hi = da.row_bytes;             // row = span bytes [mis, mis+row_bytes); whole vectors [lo,hi)
+            if (kAny) {
+                mis = (uint32_t)((uintptr_t)drow & 15u);
+                lo = (mis + 15u) & ~15u;
+                hi = (mis + da.row_bytes) & ~15u;
+                if (hi < lo) hi = lo;
+                const unsigned char* sb = smem + (size_t)buf * da.row_stride;
+                for (uint32_t o = mis; o < min(lo, mis + da.row_bytes); o += 2) *(uint16_t*)(drow - mis + o) = *(const uint16_t*)(sb + o);
+                for (uint32_t o = max(hi, mis); o < mis + da.row_bytes; o += 2) *(uint16_t*)(drow - mis + o) = *(const uint16_t*)(sb + o);
+                fence_async_smem();                                  // these reads, before the buffer is refilled by bulk copies
+            }
+            for (uint32_t off = lo; off < hi; off += kPiece)
+                bulk_store(drow - mis + off, srcb + off, min(kPiece, hi - off));
             bulk_commit();
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         };
@@ -166,14 +197,25 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
             if (aborted) break;
             if (buf) drow1 = (unsigned char*)(p.dlogits + ri.dl_offset);
             else drow0 = (unsigned char*)(p.dlogits + ri.dl_offset);
+            ri.mis = kAny ? (unsigned)((uintptr_t)row & 15u) : 0u;
+            ri.pad = 0;
             s_row[buf] = ri;
             const uint32_t dst = buf_addr + (uint32_t)buf * da.row_stride;
-            mbar_arrive_expect_tx(landed(buf, 0), head_bytes);       // release: publishes s_row[buf]
-            for (uint32_t off = 0; off < head_bytes; off += kPiece)
-                bulk_load(dst + off, row + off, min(kPiece, head_bytes - off), landed(buf, 0));
-            mbar_arrive_expect_tx(landed(buf, 1), da.row_bytes - head_bytes);
-            for (uint32_t off = head_bytes; off < da.row_bytes; off += kPiece)
-                bulk_load(dst + off, row + off, min(kPiece, da.row_bytes - off), landed(buf, 1));
+            if (kAny) {
+                // the aligned span around the row, as one part
+                const uint32_t span = (ri.mis + da.row_bytes + 15u) & ~15u;
+                mbar_arrive_expect_tx(landed(buf, 0), span);         // release: publishes s_row[buf]
+                for (uint32_t off = 0; off < span; off += kPiece)
+                    bulk_load(dst + off, row - ri.mis + off, min(kPiece, span - off), landed(buf, 0));
+                mbar_arrive_expect_tx(landed(buf, 1), 0);
+            } else {
+                mbar_arrive_expect_tx(landed(buf, 0), head_bytes);   // release: publishes s_row[buf]
+                for (uint32_t off = 0; off < head_bytes; off += kPiece)
+                    bulk_load(dst + off, row + off, min(kPiece, head_bytes - off), landed(buf, 0));
+                mbar_arrive_expect_tx(landed(buf, 1), da.row_bytes - head_bytes);
+                for (uint32_t off = head_bytes; off < da.row_bytes; off += kPiece)
+                    bulk_load(dst + off, row + off, min(kPiece, da.row_bytes - off), landed(buf, 1));
+            }
             if (rows_mine > 0) {
                 const long long target = ((i + 1) * pads_mine) / rows_mine;
                 while (pads_done < target) { zero_fill_next(); ++pads_done; }
@@ -188,8 +230,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
 
     // ---------------------------------------------------------------- consumers
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
-    const int cnt = (uint32_t)tid < nvec ? (int)((nvec - tid + kCons - 1) / kCons) : 0;   // this thread's vectors
-    const int head_cnt = min(cnt, (int)(head_vecs / kCons) + ((uint32_t)tid < head_vecs % kCons ? 1 : 0));
+    const int cnt0 = (uint32_t)tid < nvec ? (int)((nvec - tid + kCons - 1) / kCons) : 0;   // this thread's vectors
+    const int head_cnt0 = min(cnt0, (int)(head_vecs / kCons) + ((uint32_t)tid < head_vecs % kCons ? 1 : 0));
     // the block's slice of the value loss, while its first row is still on the way (thread 0 keeps the sums)
     double sum_pg = 0.0, sum_vf = 0.0;
     if (p.fused) sum_vf = consumer_sum_double<NW>(value_loss_slice(p, N, tid, kCons), s_dbl, warp, lane);
@@ -201,10 +243,28 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         mbar_wait(landed(buf, 0), use, p.status, aborted);
         RowInfo ri = s_row[buf];
         if (aborted) { ri.y = 0; ri.bad_id = 1; ri.flat = 0; }      // stale row info: touch nothing
-        const uint32_t yvec = (uint32_t)ri.y >> 3;
-        const int yj = ri.y & 7;
+        // where the row sits in the buffer: eoff entries of vector 0 precede it (kAny), vectors [0, row_vecs)
+        const uint32_t eoff = kAny ? (ri.mis >> 1) : 0u;
+        int cnt = cnt0, head_cnt = head_cnt0;
+        int jfirst = -1, jlast = -1;                               // this thread's vectors with entries outside the row
+        if (kAny) {
+            const uint32_t row_vecs = (ri.mis + da.row_bytes + 15u) >> 4;
+            cnt = (uint32_t)tid < row_vecs ? (int)((row_vecs - tid + kCons - 1) / kCons) : 0;
+            head_cnt = cnt;
+            if (eoff != 0 && tid == 0) jfirst = 0;
+            if (((eoff + (uint32_t)p.V) & 7u) != 0 && ((row_vecs - 1) % kCons) == (uint32_t)tid) jlast = (int)((row_vecs - 1) / kCons);
+        }
+        const uint32_t yvec = (eoff + (uint32_t)ri.y) >> 3;
+        const int yj = (int)((eoff + (uint32_t)ri.y) & 7u);
         const bool owner = (yvec % kCons) == (uint32_t)tid;
         const int jy = owner ? (int)(yvec / kCons) : -1;            // which of this thread's vectors holds the label
+        // one vector of this thread, with whatever is special about it
+        auto add_special = [&](Acc& acc, const uint4& q, int j, float& zy_out) {
+            if (kAny && j == jfirst) zy_out += acc_add_vec_range(acc, q, (int)eoff, 8, j == jy ? yj : -1);
+            else if (kAny && j == jlast) zy_out += acc_add_vec_range(acc, q, 0, (int)((eoff + (uint32_t)p.V) & 7u), j == jy ? yj : -1);
+            else if (j == jy) zy_out = acc_add_vec_label(acc, q, yj);
+            else acc_add_vec(acc, q);
+        };
         const uint4* src = (const uint4*)(smem + (size_t)buf * da.row_stride) + tid;
 
         // ---- pass 1: partition sum
@@ -216,12 +276,9 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 uint4 q[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) q[u] = src[(size_t)(j + u) * kCons];
-                if ((unsigned)(jy - j) < 4u) {
+                if ((unsigned)(jy - j) < 4u || (kAny && ((unsigned)(jfirst - j) < 4u || (unsigned)(jlast - j) < 4u))) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (j + u == jy) zy = acc_add_vec_label(a, q[u], yj);
-                        else acc_add_vec(a, q[u]);
-                    }
+                    for (int u = 0; u < 4; ++u) add_special(a, q[u], j + u, zy);
                 } else {
                     const float vs = exp_sum_vecs<4>(q, -a.M);
                     if (vs <= 1.8446744e19f) {
@@ -232,13 +289,9 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                     }
                 }
             }
-            for (; j < j1; ++j) {
-                const uint4 q = src[(size_t)j * kCons];
-                if (j == jy) zy = acc_add_vec_label(a, q, yj);
-                else acc_add_vec(a, q);
-            }
+            for (; j < j1; ++j) add_special(a, src[(size_t)j * kCons], j, zy);
         };
-        if (cnt > 0 && jy != 0) a.M = max8_scaled(src[0]);          // this thread's reference exponent for the row
+        if (cnt > 0 && jy != 0 && jfirst != 0 && jlast != 0) a.M = max8_scaled(src[0]);          // this thread's reference exponent for the row
         sum_range(0, head_cnt);
         mbar_wait(landed(buf, 1), use, p.status, aborted);
         sum_range(head_cnt, cnt);

@@ -313,6 +313,8 @@ def test_gpt2_vocabulary_rows_off_16_byte_boundaries(oracle):
     batch["actor"][0, 0, 0], batch["actor"][0, 1, w.V - 1], batch["actor"][1, 0, 7] = 4.0, 4.0, 4.0
     run = OracleRun(oracle, w, batch)
     out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+    dlogits_properties(run, out, batch["ids"], batch["actor"])
+    run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], in_place=True, all_rows=True)
     _experience_both_ways(w, batch, batch["actor"], batch["ref"], batch["ids"])
     # a view that starts in the middle of a row of a larger tensor: odd base address as well
     big = torch.zeros((3, 12, w.V + 5), dtype=torch.bfloat16, device=DEV)
@@ -321,3 +323,14 @@ def test_gpt2_vocabulary_rows_off_16_byte_boundaries(oracle):
     ws = binding.workspace(w.B, w.T, DEV)
     lp = binding.gather_logprobs(view, batch["ids"], batch["lengths"], ws)
     assert np.abs(np32(lp).astype(np.float64) - run.lp_actor).max() <= TOL_LP
+    # the loss in place on that view: the 3 + 2 entries either side of every row must stay untouched
+    big[:, :, :3] = 7.0
+    big[:, :, 3 + w.V:] = -7.0
+    run_steps(oracle, w, batch, run, view, batch["ref"], batch["ids"], all_rows=True)      # out of place, other layout
+    t = lambda a: torch.as_tensor(a, device=DEV)
+    outp = binding.PPOOutputs(view, in_place=True)
+    binding.ppo_loss_fwd_bwd(view, batch["ids"], batch["lengths"], t(run.lp_old_in), t(run.adv_in), t(run.values_new_in),
+                             t(run.values_old_in), t(run.ret_in), w.clip_eps, w.value_clip, run.grad_scale, ws, outp)
+    assert binding.poll_status(ws) == 0
+    assert (big[:, :, :3] == 7.0).all() and (big[:, :, 3 + w.V:] == -7.0).all()
+    check_dlogits_rows(oracle, run, batch["actor"], batch["ids"], view, np.arange(w.B * w.T))
