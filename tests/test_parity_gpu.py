@@ -334,3 +334,36 @@ def test_gpt2_vocabulary_rows_off_16_byte_boundaries(oracle):
     assert binding.poll_status(ws) == 0
     assert (big[:, :, :3] == 7.0).all() and (big[:, :, 3 + w.V:] == -7.0).all()
     check_dlogits_rows(oracle, run, batch["actor"], batch["ids"], view, np.arange(w.B * w.T))
+
+
+@pytest.mark.parametrize("V", [1000, 50272, 1001])
+def test_device_detected_errors_are_flagged_not_faulted(oracle, V):
+    # an id outside the vocabulary and lengths outside [0,T]: status flags, the offending token's outputs are 0,
+    # everything else is computed as if the lengths had been clamped
+    w = inputs.scaled(inputs.WORKLOADS["tiny"], V=V, B=3, T=8, lengths="full", seed=3)
+    batch = inputs.make_batch(w, device=DEV)
+    ws = binding.workspace(w.B, w.T, DEV)
+    good = OracleRun(oracle, w, batch)
+    bad_ids = batch["ids"].clone()
+    bad_ids[1, 2] = V
+    bad_ids[2, 5] = -1
+    lp = binding.gather_logprobs(batch["actor"], bad_ids, batch["lengths"], ws)
+    assert binding.poll_status(ws) == 16 and binding.poll_status(ws) == 0          # reported once, then cleared
+    got = np32(lp).astype(np.float64)
+    assert got[1, 2] == 0 and got[2, 5] == 0
+    mask = np.ones((3, 8), bool); mask[1, 2] = mask[2, 5] = False
+    assert np.abs(got - good.lp_actor)[mask].max() <= TOL_LP
+    # lengths: 99 is clamped to T, -4 to 0
+    bad_len = torch.tensor([99, -4, 8], dtype=torch.int32, device=DEV)
+    lp = binding.gather_logprobs(batch["actor"], batch["ids"], bad_len, ws)
+    assert binding.poll_status(ws) == 32
+    got = np32(lp).astype(np.float64)
+    assert np.abs(got[0] - good.lp_actor[0]).max() <= TOL_LP and (got[1] == 0).all()
+    # both at once in the loss: flags are OR-ed; the bad token's gradient row is zero
+    out = binding.PPOOutputs(batch["actor"])
+    f = lambda a: torch.as_tensor(a, device=DEV)
+    binding.ppo_loss_fwd_bwd(batch["actor"], bad_ids, bad_len, f(good.lp_old_in), f(good.adv_in), f(good.values_new_in),
+                             f(good.values_old_in), f(good.ret_in), w.clip_eps, w.value_clip, 1.0, ws, out)
+    assert binding.poll_status(ws) == (16 | 32)
+    assert (out.dlogits[2, 5].view(torch.int16) == 0).all() and (out.dlogits[1].view(torch.int16) == 0).all()
+    assert torch.isfinite(out.loss).all() and torch.isfinite(out.dlogits.float()).all()
