@@ -85,12 +85,12 @@ bool rows_16B(const void* base, long long stride_b, long long stride_t, int V)
     return aligned(base, 16) && (stride_b % 8) == 0 && (stride_t % 8) == 0 && (V % 8) == 0;
 }
 
-template <bool kLoss, int NW, int U>
+template <int NW, int U>
 int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_t s)
 {
-    RLHF_CUDA(cudaFuncSetAttribute(row_ring_kernel<kLoss, NW, U>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RLHF_CUDA(cudaFuncSetAttribute(row_ring_kernel<NW, U>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)pl.smem_bytes));
-    row_ring_kernel<kLoss, NW, U><<<grid, NW * 32 + 32, pl.smem_bytes, s>>>(ra);
+    row_ring_kernel<NW, U><<<grid, NW * 32 + 32, pl.smem_bytes, s>>>(ra);
     return RLHF_OK;
 }
 
@@ -133,14 +133,12 @@ int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     return RLHF_OK;
 }
 
-template <bool kLoss>
-int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
+// The loss row kernel for 16-byte aligned rows: two resident rows where that fits, else the chunk ring.
+int launch_loss_rows(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 {
     const unsigned row_bytes = 2u * (unsigned)a.V;
-    if constexpr (kLoss) {
-        if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false>(a, dev, s);
-    }
-    const RingPlan pl = plan_ring(row_bytes, kLoss, dev.smem_per_sm, dev.max_smem_optin);
+    if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false>(a, dev, s);
+    const RingPlan pl = plan_ring(row_bytes, dev.smem_per_sm, dev.max_smem_optin);
     RingArgs ra{};
     ra.row = a;
     ra.n_slots = pl.n_slots;
@@ -149,11 +147,9 @@ int launch_ring(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     ra.row_bytes = row_bytes;
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * pl.blocks_per_sm);
-    if constexpr (kLoss) {
-        if (pl.NW == 16) return launch_ring_as<true, 16, 2>(ra, pl, grid, s);
-    }
-    if (pl.U == 1) return launch_ring_as<kLoss, 8, 1>(ra, pl, grid, s);
-    return launch_ring_as<kLoss, 8, 2>(ra, pl, grid, s);
+    if (pl.NW == 16) return launch_ring_as<16, 2>(ra, pl, grid, s);
+    if (pl.U == 1) return launch_ring_as<8, 1>(ra, pl, grid, s);
+    return launch_ring_as<8, 2>(ra, pl, grid, s);
 }
 
 // The row kernels run with the largest shared-memory carve-out.  A kernel that prefers another
@@ -453,7 +449,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
         if (ragged_fast) {
             if (int e = launch_dbuf<true>(a, dev, s)) return e;
         } else {
-            if (int e = launch_ring<true>(a, dev, s)) return e;
+            if (int e = launch_loss_rows(a, dev, s)) return e;
         }
         return launch_check("loss row kernel");
     } else {

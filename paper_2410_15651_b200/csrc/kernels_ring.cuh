@@ -1,18 +1,19 @@
-// Fast row kernels for 16-byte aligned rows (sm_100a).
+// Loss row kernel with a ring of shared-memory chunks, for 16-byte aligned rows outside the range of
+// the two-resident-rows kernel (sm_100a); also the PTX wrappers and per-vector arithmetic that the
+// other row kernels share.
 //
-// Each persistent block owns a ring of shared-memory slots.  One elected producer thread streams
-// the block's rows into the ring with bulk asynchronous copies (cp.async.bulk, completion counted
-// on an mbarrier per slot); 8 consumer warps reduce the slots as they land.  HBM latency is
-// covered by the bytes the ring keeps in flight, not by registers or occupancy.
+// Each persistent block owns a ring of 4/8/16 KB slots.  One elected producer thread streams the
+// block's rows into the ring with bulk asynchronous copies (cp.async.bulk, completion counted on an
+// mbarrier per slot); NW consumer warps work on the slots as they land and release them through a
+// second mbarrier per slot.
 //
-//   log-prob kernel   every slot is released as soon as it has been summed (streaming).
-//   loss kernel       if a whole row fits in the ring ("resident"), the row is summed as it lands,
-//                     kept, and then turned into dlogits straight from shared memory, so that DRAM
-//                     sees one read and one write per row; slots are released chunk by chunk in
-//                     the second pass and refilled with the next row at once.  Rows larger than
-//                     the ring are streamed twice (the second read is served by L2).
-//                     Padded rows are zero-filled by bulk stores from a zeroed shared buffer,
-//                     issued by the producer thread between its loads.
+//   short rows (< 16 KB)     blocks of 8 consumer warps, up to 7 per SM; the row stays in the ring
+//                            ("resident") between the partition-sum pass and the gradient pass.
+//   rows of 111 KB .. 225 KB one block of 16 consumer warps per SM, row resident.
+//   larger rows              streamed twice by one block of 16 consumer warps per SM; the second read
+//                            is served by L2.
+//   Padded rows are zero-filled by bulk stores from a zeroed shared buffer, issued by the producer
+//   thread between its loads.
 //
 // Work assignment is static: block i takes valid rows i, i+G, i+2G, ... (and padded rows likewise),
 // so results never depend on timing.  Every wait on an mbarrier is bounded; if one runs out the
@@ -263,8 +264,8 @@ __device__ __forceinline__ float max8_scaled(const uint4& q)
 
 // Dynamic shared memory: [n_slots * chunk][full barriers n_slots * 8][empty barriers n_slots * 8][zero buffer].
 // NW consumer warps + 1 producer warp; a chunk is NW*32*U 16-byte vectors.
-template <bool kLoss, int NW, int U>
-__global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) row_ring_kernel(RingArgs ra)
+template <int NW, int U>
+__global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kernel(RingArgs ra)
 {
     constexpr int kCons = NW * 32;
     constexpr int kThreads = kCons + 32;
@@ -294,10 +295,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
         }
         fence_mbar_init();
     }
-    if (kLoss) {
-        for (int i = tid; i < kZeroBytes / 16; i += kThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
-        fence_async_smem();
-    }
+    for (int i = tid; i < kZeroBytes / 16; i += kThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
+    fence_async_smem();
     __syncthreads();
 
     bool aborted = false;
@@ -307,7 +306,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
         if (lane != 0) return;
         const long long n_pad = (long long)p.B * p.T - N;
         const long long rows_mine = N > blockIdx.x ? (N - blockIdx.x + G - 1) / G : 0;
-        const long long pads_mine = (kLoss && n_pad > blockIdx.x) ? (n_pad - blockIdx.x + G - 1) / G : 0;
+        const long long pads_mine = (n_pad > blockIdx.x) ? (n_pad - blockIdx.x + G - 1) / G : 0;
         Cursor cur{0, 0}, pcur{0, 0};
         long long pads_done = 0;
         auto zero_fill_next = [&]() {
@@ -320,7 +319,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
         };
         int slot = 0;
         uint32_t phase = 0;
-        const int loads_per_row = (kLoss && !ra.resident) ? 2 * chunks : chunks;
+        const int loads_per_row = (!ra.resident) ? 2 * chunks : chunks;
         long long i = 0;
         for (long long k = blockIdx.x; k < N && !aborted; k += G, ++i) {
             int b, t;
@@ -336,32 +335,22 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
                 bulk_load(slots_addr + (uint32_t)slot * kChunk, row + off, bytes, full_addr + 8u * slot);
                 if (++slot == S) { slot = 0; phase ^= 1u; }
             }
-            if (kLoss) {
+            {
                 const long long target = ((i + 1) * pads_mine) / rows_mine;
                 while (pads_done < target) { zero_fill_next(); ++pads_done; }
             }
         }
-        if (kLoss) {
-            while (pads_done < pads_mine) { zero_fill_next(); ++pads_done; }
-            bulk_wait_all();
-        }
+        while (pads_done < pads_mine) { zero_fill_next(); ++pads_done; }
+        bulk_wait_all();
         return;
     }
 
     // ---------------------------------------------------------------- consumers
-    if (!kLoss) {
-        // log-prob 0 at padded tokens
-        const long long total = (long long)p.B * p.T;
-        for (long long i = (long long)blockIdx.x * kCons + tid; i < total; i += G * kCons) {
-            int b = (int)(i / p.T), t = (int)(i % p.T);
-            if (t >= clamp_len(__ldg(p.lengths + b), p.T)) p.out_lp[i] = 0.f;
-        }
-    }
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
     const uint32_t nvec = ra.row_bytes / 16u;
     const int full_chunks = (int)(nvec / kChunkVecs);          // chunks in which every vector exists
     double sum_pg = 0.0, sum_vf = 0.0;                         // block partial sums (thread 0)
-    if (kLoss && p.fused) sum_vf = consumer_sum_double<NW>(value_loss_slice(p, N, tid, kCons), s_dbl, warp, lane);
+    if (p.fused) sum_vf = consumer_sum_double<NW>(value_loss_slice(p, N, tid, kCons), s_dbl, warp, lane);
 
     Cursor cur{0, 0};
     int slot = 0;
@@ -375,11 +364,9 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
     auto fetch_row = [&](long long k) {
         if (k < N && cursor_seek_valid(cur, k, p.lengths, p.B, p.T, nb, nt)) {
             ny = __ldg(p.ids + (long long)nb * p.ids_stride_b + nt);
-            if (kLoss) {
-                const long long f = (long long)nb * p.T + nt;
-                n_lp_old = __ldg(p.lp_old + f);
-                n_adv = __ldg(p.adv + f);
-            }
+            const long long f = (long long)nb * p.T + nt;
+            n_lp_old = __ldg(p.lp_old + f);
+            n_adv = __ldg(p.adv + f);
         }
     };
     fetch_row(blockIdx.x);
@@ -431,7 +418,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
                     }
                 }
             }
-            if (!(kLoss && ra.resident)) {
+            if (!ra.resident) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty_addr + 8u * slot);
             }
@@ -443,11 +430,6 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
 
         // scalars of the next row, in flight while this row is finished
         fetch_row(k + G);
-
-        if (!kLoss) {
-            if (tid == 0) p.out_lp[flat] = bad_id ? 0.f : r.lp;
-            continue;
-        }
 
         float loss = 0.f, g = 0.f;
         if (!bad_id) ppo_token(r.lp, lp_old, adv, p.clip_eps, scale_over_N, loss, g);
@@ -492,7 +474,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, kLoss ? (NW == 16 ? 1 : 3) : 4) 
             if (++slot == S) { slot = 0; phase ^= 1u; }
         }
     }
-    if (kLoss && p.fused && tid == 0) publish_block_losses(p, N, sum_pg, sum_vf);
+    if (p.fused && tid == 0) publish_block_losses(p, N, sum_pg, sum_vf);
 }
 
 // ---------------------------------------------------------------- host-side plan
@@ -506,31 +488,31 @@ struct RingPlan {
     size_t smem_bytes = 0;
 };
 
-inline size_t ring_smem_bytes(int NW, int U, int n_slots, bool loss)
+inline size_t ring_smem_bytes(int NW, int U, int n_slots)
 {
-    return (size_t)n_slots * ((size_t)NW * 32 * 16 * U) + (size_t)n_slots * 16 + (loss ? kZeroBytes : 0);
+    return (size_t)n_slots * ((size_t)NW * 32 * 16 * U) + (size_t)n_slots * 16 + kZeroBytes;
 }
 
 // Chooses block shape, chunk size, ring depth and blocks per SM for rows of `row_bytes`.
 // sm_smem: shared memory per SM; block_smem_max: opt-in maximum per block.  The system reserves
 // 1 KB per resident block.
-inline RingPlan plan_ring(unsigned row_bytes, bool loss, int sm_smem, int block_smem_max)
+inline RingPlan plan_ring(unsigned row_bytes, int sm_smem, int block_smem_max)
 {
     constexpr size_t kStatic = 1280;                   // static shared memory of the kernel, rounded up
     constexpr size_t kReserved = 1024;
-    if (loss && row_bytes >= 32768) {
+    if (row_bytes >= 32768) {
         // long rows that fit: one block of 16 consumer warps per SM owns all of its shared memory, in
         // 16 KB chunks; the ring holds the row being processed plus as much of the next as fits, so
         // loads keep streaming while a row is reduced.
         const int NW = 16, U = 2;
         const size_t chunk = (size_t)NW * 32 * 16 * U;
         const int chunks = (int)((row_bytes + chunk - 1) / chunk);
-        if (ring_smem_bytes(NW, U, chunks, true) + kStatic <= (size_t)block_smem_max) {
+        if (ring_smem_bytes(NW, U, chunks) + kStatic <= (size_t)block_smem_max) {
             int S = chunks;
-            while (ring_smem_bytes(NW, U, S + 1, true) + kStatic <= (size_t)block_smem_max) ++S;
-            return RingPlan{NW, U, S, chunks, 1, 1, ring_smem_bytes(NW, U, S, true)};
+            while (ring_smem_bytes(NW, U, S + 1) + kStatic <= (size_t)block_smem_max) ++S;
+            return RingPlan{NW, U, S, chunks, 1, 1, ring_smem_bytes(NW, U, S)};
         }
-    } else if (loss) {
+    } else {
         // short rows: blocks of 8 consumer warps, as many per SM as can hold a row each (at most 7 by
         // thread count); among chunk sizes that reach that count take the preferred one; the ring then
         // grows into what is left.
@@ -541,34 +523,26 @@ inline RingPlan plan_ring(unsigned row_bytes, bool loss, int sm_smem, int block_
         for (int U : order) {
             const size_t chunk = (size_t)NW * 32 * 16 * U;
             const int chunks = (int)((row_bytes + chunk - 1) / chunk);
-            const size_t need = ring_smem_bytes(NW, U, chunks, true) + kStatic;
+            const size_t need = ring_smem_bytes(NW, U, chunks) + kStatic;
             if (need > (size_t)block_smem_max) continue;
             int k = (int)std::min<size_t>(kMaxBlocksByThreads, (size_t)sm_smem / (need + kReserved));
             if (k < 1 || k <= best.blocks_per_sm) continue;
             const size_t per_block = std::min<size_t>((size_t)sm_smem / k - kReserved, (size_t)block_smem_max) - kStatic;
             int S = chunks;
-            while (ring_smem_bytes(NW, U, S + 1, true) <= per_block) ++S;
-            best = RingPlan{NW, U, S, chunks, 1, k, ring_smem_bytes(NW, U, S, true)};
+            while (ring_smem_bytes(NW, U, S + 1) <= per_block) ++S;
+            best = RingPlan{NW, U, S, chunks, 1, k, ring_smem_bytes(NW, U, S)};
         }
         if (best.NW) return best;
     }
-    if (loss) {
-        // rows larger than shared memory are streamed twice.  One block of 16 consumer warps per SM
-        // keeps the number of rows in flight at the number of SMs, so that the second read of a row
-        // (a few tens of microseconds after the first) is still served by L2.
-        const int NW = 16, U = 2;
-        const size_t chunk = (size_t)NW * 32 * 16 * U;
-        const int chunks = (int)((row_bytes + chunk - 1) / chunk);
-        int S = 2;
-        while (ring_smem_bytes(NW, U, S + 1, true) + kStatic <= (size_t)block_smem_max) ++S;
-        return RingPlan{NW, U, S, chunks, 0, 1, ring_smem_bytes(NW, U, S, true)};
-    }
-    // log-prob streaming (not used by the warp-per-row kernel): 4 blocks of 8 consumer warps per SM
-    const int NW = 8, U = row_bytes > 4096 ? 2 : 1;
+    // rows larger than shared memory are streamed twice.  One block of 16 consumer warps per SM
+    // keeps the number of rows in flight at the number of SMs, so that the second read of a row
+    // (a few tens of microseconds after the first) is still served by L2.
+    const int NW = 16, U = 2;
     const size_t chunk = (size_t)NW * 32 * 16 * U;
     const int chunks = (int)((row_bytes + chunk - 1) / chunk);
-    const int S = (int)((48 * 1024) / chunk);
-    return RingPlan{NW, U, S, chunks, 0, 4, ring_smem_bytes(NW, U, S, loss)};
+    int S = 2;
+    while (ring_smem_bytes(NW, U, S + 1) + kStatic <= (size_t)block_smem_max) ++S;
+    return RingPlan{NW, U, S, chunks, 0, 1, ring_smem_bytes(NW, U, S)};
 }
 
 }  // namespace rlhf
