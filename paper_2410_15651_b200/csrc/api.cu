@@ -85,12 +85,30 @@ bool rows_16B(const void* base, long long stride_b, long long stride_t, int V)
     return aligned(base, 16) && (stride_b % 8) == 0 && (stride_t % 8) == 0 && (V % 8) == 0;
 }
 
+// Launches `kernel` with programmatic stream serialisation allowed (see pdl_wait_prior_grid): the launch
+// itself and the kernel's set-up overlap the tail of the kernel before it in the stream.
+template <typename... Params, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 template <int NW, int U>
 int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_t s)
 {
     RLHF_CUDA(cudaFuncSetAttribute(row_ring_kernel<NW, U>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)pl.smem_bytes));
-    row_ring_kernel<NW, U><<<grid, NW * 32 + 32, pl.smem_bytes, s>>>(ra);
+    RLHF_CUDA(launch_kernel(row_ring_kernel<NW, U>, grid, NW * 32 + 32, pl.smem_bytes, s, ra));
     return RLHF_OK;
 }
 
@@ -106,7 +124,7 @@ int launch_warp_logprob(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
     RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps, kDual, kAny>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    logprob_warp_kernel<kLogprobWarps, kDual, kAny><<<grid, kLogprobWarps * 32, smem, s>>>(wa);
+    RLHF_CUDA(launch_kernel(logprob_warp_kernel<kLogprobWarps, kDual, kAny>, grid, kLogprobWarps * 32, smem, s, wa));
     return RLHF_OK;
 }
 
@@ -129,7 +147,7 @@ int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
     RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps, kAny>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    loss_dbuf_kernel<kDbufWarps, kAny><<<grid, kDbufWarps * 32 + 32, smem, s>>>(da);
+    RLHF_CUDA(launch_kernel(loss_dbuf_kernel<kDbufWarps, kAny>, grid, kDbufWarps * 32 + 32, smem, s, da));
     return RLHF_OK;
 }
 
@@ -285,8 +303,8 @@ int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score,
     long long total = (long long)B * T;
     int grid = (int)std::min<long long>((total + 255) / 256, 1184);
     if (int e = keep_max_carveout(kl_reward_kernel)) return e;
-    kl_reward_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(lp_old, lp_ref, score, lengths, B, T,
-                                                           beta_kl, reward_clip, out_rewards);
+    RLHF_CUDA(launch_kernel(kl_reward_kernel, grid, 256, 0, (cudaStream_t)stream, lp_old, lp_ref, score, lengths, B, T,
+                            beta_kl, reward_clip, out_rewards));
     return launch_check("kl_reward_kernel");
 }
 
@@ -304,8 +322,8 @@ int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, 
         return RLHF_ERR_STRIDE;
     int grid = (B + kGaeWarpsPerBlock - 1) / kGaeWarpsPerBlock;
     if (int e = keep_max_carveout(gae_kernel)) return e;
-    gae_kernel<<<grid, kGaeWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(rewards, values_old, lengths, B, T,
-                                                                       gamma, lambda, out_adv, out_returns);
+    RLHF_CUDA(launch_kernel(gae_kernel, grid, kGaeWarpsPerBlock * 32, 0, (cudaStream_t)stream, rewards, values_old,
+                            lengths, B, T, gamma, lambda, out_adv, out_returns));
     return launch_check("gae_kernel");
 }
 
@@ -369,9 +387,9 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     if (int e = launch_check("logprob_warp_kernel<dual>")) return e;
     if (int e = keep_max_carveout(reward_gae_kernel)) return e;
     const int grid = (B + kGaeWarpsPerBlock - 1) / kGaeWarpsPerBlock;
-    reward_gae_kernel<<<grid, kGaeWarpsPerBlock * 32, 0, s>>>(lp_old ? lp_old : out_lp_actor, out_lp_ref, score,
-                                                             values_old, lengths, B, T, beta_kl, reward_clip,
-                                                             gamma, lambda, out_rewards, out_adv, out_returns);
+    RLHF_CUDA(launch_kernel(reward_gae_kernel, grid, kGaeWarpsPerBlock * 32, 0, s, lp_old ? lp_old : out_lp_actor,
+                            out_lp_ref, score, values_old, lengths, B, T, beta_kl, reward_clip, gamma, lambda,
+                            out_rewards, out_adv, out_returns));
     return launch_check("reward_gae_kernel");
 }
 
@@ -454,7 +472,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
         return launch_check("loss row kernel");
     } else {
         int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
-        row_generic_kernel<true><<<grid, kGenericThreads, 0, s>>>(a);
+        RLHF_CUDA(launch_kernel(row_generic_kernel<true>, grid, kGenericThreads, 0, s, a));
         if (int e = launch_check("row_generic_kernel<loss>")) return e;
     }
 
@@ -476,7 +494,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
     f.partials = (double*)(ws + kPartialsOffset);
     int fgrid = (int)std::min<long long>((rows + 1023) / 1024, kFinalMaxBlocks);
     if (int e = keep_max_carveout(ppo_finalize_kernel)) return e;
-    ppo_finalize_kernel<<<fgrid, kFinalThreads, 0, s>>>(f);
+    RLHF_CUDA(launch_kernel(ppo_finalize_kernel, fgrid, kFinalThreads, 0, s, f));
     return launch_check("ppo_finalize_kernel");
 }
 

@@ -22,6 +22,8 @@
 
 namespace rlhf {
 
+constexpr long long kTailPads = 2;      // padded rows of a block that are zero-filled after its last load
+
 struct DbufArgs {
     RowArgs row;
     unsigned row_bytes;     // 2*V, multiple of 16
@@ -114,9 +116,6 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     const uint32_t head_vecs = nvec >= 8u * kCons ? 4u * kCons : nvec;
     const uint32_t head_bytes = head_vecs * 16u;
 
-    const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
-    const long long G = gridDim.x;
-
     if (tid == 0) {
         for (int i = 0; i < 4; ++i) mbar_init(bar_addr + 8u * i, 1);
         mbar_init(computed(0), NW);
@@ -126,6 +125,11 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     for (int i = tid; i < kZeroBytes / 16; i += kThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
     __syncthreads();
+    pdl_wait_prior_grid();                       // nothing above touches global memory
+    pdl_release_next_grid();
+
+    const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
+    const long long G = gridDim.x;
 
     bool aborted = false;
 
@@ -134,12 +138,16 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         if (lane != 0) return;
         const long long n_pad = (long long)p.B * p.T - N;
         const long long rows_mine = N > blockIdx.x ? (N - blockIdx.x + G - 1) / G : 0;
-        const long long pads_mine = n_pad > blockIdx.x ? (n_pad - blockIdx.x + G - 1) / G : 0;
+        const PadShare pads = pad_share(N, n_pad, G, blockIdx.x);
+        const long long pads_mine = pads.count;
+        // the last padded rows are kept back until the block's last valid row has been requested: their
+        // stores then keep the memory pipe busy while that row is still being reduced
+        const long long pads_early = pads_mine > kTailPads ? pads_mine - kTailPads : 0;
         Cursor cur{0, 0}, pcur{0, 0};
         long long pads_done = 0;
         auto zero_fill_next = [&]() {
             int b, t;
-            if (!cursor_seek_padded(pcur, blockIdx.x + pads_done * G, p.lengths, p.B, p.T, b, t)) return;
+            if (!cursor_seek_padded(pcur, pads.start + pads_done, p.lengths, p.B, p.T, b, t)) return;
             unsigned char* drow = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t);
             uint32_t lo = 0, hi = da.row_bytes;                  // [lo,hi): the part of the row made of whole 16-byte vectors
             if (kAny) {
@@ -217,7 +225,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                     bulk_load(dst + off, row + off, min(kPiece, da.row_bytes - off), landed(buf, 1));
             }
             if (rows_mine > 0) {
-                const long long target = ((i + 1) * pads_mine) / rows_mine;
+                const long long target = ((i + 1) * pads_early) / rows_mine;
                 while (pads_done < target) { zero_fill_next(); ++pads_done; }
             }
         }
@@ -321,8 +329,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
 #pragma unroll
                 for (int u = 0; u < 4; ++u) q[u] = src[(size_t)(j + u) * kCons];
                 uint4 o[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) o[u] = grad_vec(q[u], c2, sign2);
+                grad_vecs<4>(q, o, c2, sign2);
                 if ((unsigned)(jy - j) < 4u) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u)

@@ -59,6 +59,8 @@ __global__ void __launch_bounds__(kGenericThreads) row_generic_kernel(RowArgs p)
 {
     __shared__ Acc s_acc[32];
     __shared__ long long s_cnt[33];
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
 

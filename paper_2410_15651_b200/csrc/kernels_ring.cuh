@@ -171,19 +171,42 @@ __device__ __forceinline__ float acc_add_vec_range(Acc& a, const uint4& q, int j
     return zy;
 }
 
-// dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.
+#ifndef RLHF_POLY_MASKS
+#define RLHF_POLY_MASKS 0x0, 0x0, 0x0
+#endif
+constexpr int kPolyMasks[3] = {RLHF_POLY_MASKS};
+constexpr int kSumPolyWords = kPolyMasks[0], kGradPolyEven = kPolyMasks[1], kGradPolyOdd = kPolyMasks[2];
+
+// dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.  kPolyWords: bit k set = entries 2k, 2k+1
+// take the FMA-pipe exponential (degree 3) instead of ex2.
+template <int kPolyWords>
+__device__ __forceinline__ uint4 grad_vec_mix(const uint4& q, float c2, uint32_t sign2)
+{
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    uint32_t o[4];
+    uint32_t seen = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 x = __ffma2_rn(unpack_bf16x2(w[k]), splat2(kLog2e), splat2(c2));
+        const float2 d = ((kPolyWords >> k) & 1) ? ex2_fma_pair<3>(x, seen) : make_float2(ex2(x.x), ex2(x.y));
+        o[k] = pack_bf16x2(d.x, d.y) ^ sign2;
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// One vector on its own: a quarter of the entries on the FMA pipe.
 __device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sign2)
 {
-    float z[8], d[8];
-    unpack8(q, z);
+    return grad_vec_mix<kGradPolyEven>(q, c2, sign2);
+}
+
+// U vectors: 3 of every 8 exponentials on the FMA pipe (1 word of even vectors, 2 of odd ones), the
+// mix at which the special-function unit and the issue slots are about equally loaded.
+template <int U>
+__device__ __forceinline__ void grad_vecs(const uint4 (&q)[U], uint4 (&o)[U], float c2, uint32_t sign2)
+{
 #pragma unroll
-    for (int i = 0; i < 8; ++i) d[i] = ex2(fmaf(z[i], kLog2e, c2));
-    uint4 o;
-    o.x = pack_bf16x2(d[0], d[1]) ^ sign2;
-    o.y = pack_bf16x2(d[2], d[3]) ^ sign2;
-    o.z = pack_bf16x2(d[4], d[5]) ^ sign2;
-    o.w = pack_bf16x2(d[6], d[7]) ^ sign2;
-    return o;
+    for (int u = 0; u < U; ++u) o[u] = (u & 1) ? grad_vec_mix<kGradPolyOdd>(q[u], c2, sign2) : grad_vec_mix<kGradPolyEven>(q[u], c2, sign2);
 }
 
 __device__ __forceinline__ void patch_label(uint4& o, int j, float value)
@@ -239,19 +262,27 @@ __device__ __forceinline__ Acc consumer_reduce(const Acc& a, float2* s_part, con
 }
 
 // ---------------------------------------------------------------- the kernel
-// Sum of the exponentials of U vectors against one reference exponent (no range check).
+// Sum of the exponentials of U vectors against one reference exponent.  A quarter of them (the last
+// word of every vector) is evaluated on the FMA pipe (degree 4).  No range handling: if an entry is 2^128
+// or more above the reference the result is +inf, and the caller, which redoes any block whose sum
+// exceeds 2^64, takes the careful path.
 template <int U>
 __device__ __forceinline__ float exp_sum_vecs(const uint4 (&q)[U], float negM)
 {
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    uint32_t seen = kPolyMagicBits;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        float z[8];
-        unpack8(q[u], z);
+        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i & 3] += ex2(fmaf(z[i], kLog2e, negM));
+        for (int k = 0; k < 4; ++k) {
+            const float2 x = __ffma2_rn(unpack_bf16x2(w[k]), splat2(kLog2e), splat2(negM));
+            const float2 e = ((kSumPolyWords >> k) & 1) ? ex2_fma_pair<4>(x, seen) : make_float2(ex2(x.x), ex2(x.y));
+            acc[k & 1] = __fadd2_rn(acc[k & 1], e);
+        }
     }
-    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    const float vs = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
+    return ex2_fma_in_range(seen) ? vs : __int_as_float(0x7f800000);
 }
 
 __device__ __forceinline__ float max8_scaled(const uint4& q)
@@ -285,9 +316,6 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
     const uint32_t empty_addr = full_addr + (uint32_t)S * 8u;
     unsigned char* zero_buf = smem + (size_t)S * kChunk + (size_t)S * 16;
 
-    const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
-    const long long G = gridDim.x;
-
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(full_addr + 8u * s, 1);
@@ -298,6 +326,11 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
     for (int i = tid; i < kZeroBytes / 16; i += kThreads) ((uint4*)zero_buf)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
     __syncthreads();
+    pdl_wait_prior_grid();                       // nothing above touches global memory
+    pdl_release_next_grid();
+
+    const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
+    const long long G = gridDim.x;
 
     bool aborted = false;
 
@@ -306,12 +339,13 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
         if (lane != 0) return;
         const long long n_pad = (long long)p.B * p.T - N;
         const long long rows_mine = N > blockIdx.x ? (N - blockIdx.x + G - 1) / G : 0;
-        const long long pads_mine = (n_pad > blockIdx.x) ? (n_pad - blockIdx.x + G - 1) / G : 0;
+        const PadShare pads = pad_share(N, n_pad, G, blockIdx.x);
+        const long long pads_mine = pads.count;
         Cursor cur{0, 0}, pcur{0, 0};
         long long pads_done = 0;
         auto zero_fill_next = [&]() {
             int b, t;
-            if (!cursor_seek_padded(pcur, blockIdx.x + pads_done * G, p.lengths, p.B, p.T, b, t)) return;
+            if (!cursor_seek_padded(pcur, pads.start + pads_done, p.lengths, p.B, p.T, b, t)) return;
             unsigned char* drow = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t);
             for (uint32_t off = 0; off < ra.row_bytes; off += kZeroBytes)
                 bulk_store(drow + off, smem_u32(zero_buf), min((uint32_t)kZeroBytes, ra.row_bytes - off));
@@ -452,8 +486,10 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
                 uint4 q[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) q[u] = src[u * kCons];
+                uint4 o[U];
+                grad_vecs<U>(q, o, c2, sign2);
 #pragma unroll
-                for (int u = 0; u < U; ++u) store_v4(dst + (size_t)u * kCons * 16, grad_vec(q[u], c2, sign2));
+                for (int u = 0; u < U; ++u) store_v4(dst + (size_t)u * kCons * 16, o[u]);
             } else {
                 const uint32_t v0 = (uint32_t)c * kChunkVecs + tid;
 #pragma unroll

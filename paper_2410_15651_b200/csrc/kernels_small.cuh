@@ -22,6 +22,8 @@ __global__ void __launch_bounds__(256) kl_reward_kernel(const float* __restrict_
                                                         const int* __restrict__ lengths, int B, int T,
                                                         float beta, float clip, float* out)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     const long long total = (long long)B * T;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -90,6 +92,8 @@ __global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) gae_kernel(const float
                                                                      float* __restrict__ adv,
                                                                      float* __restrict__ ret)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * kGaeWarpsPerBlock + (threadIdx.x >> 5);
     if (b >= B) return;
@@ -111,6 +115,8 @@ __global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) reward_gae_kernel(cons
                                                                             float* rewards, float* __restrict__ adv,
                                                                             float* __restrict__ ret)
 {
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * kGaeWarpsPerBlock + (threadIdx.x >> 5);
     if (b >= B) return;
@@ -152,6 +158,8 @@ __global__ void __launch_bounds__(kFinalThreads) ppo_finalize_kernel(FinalArgs p
     __shared__ long long s_cnt[33];
     __shared__ double s_red[2][kFinalThreads / 32];
     __shared__ bool s_last;
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
     const long long N = block_count_valid(p.lengths, p.B, p.T, s_cnt, nullptr);
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
 

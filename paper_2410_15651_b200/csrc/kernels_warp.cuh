@@ -63,11 +63,13 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
     const uint32_t ring_addr = smem_u32(ring);
     const uint32_t bar_addr = smem_u32(smem + (size_t)WPB * (kWarpSlots * kWarpChunk)) + (uint32_t)warp * (kWarpSlots * 8);
 
-    const int N1 = (int)block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
     if (lane == 0) {
         for (int s = 0; s < kWarpSlots; ++s) mbar_init(bar_addr + 8u * s, 1);
         fence_mbar_init();
     }
+    pdl_wait_prior_grid();                       // nothing above touches global memory
+    pdl_release_next_grid();
+    const int N1 = (int)block_count_valid(p.lengths, p.B, p.T, s_cnt, blockIdx.x == 0 ? p.status : nullptr);
     __syncthreads();
 
     // log-prob 0 at padded tokens

@@ -57,6 +57,11 @@ def run_steps(oracle, w, batch, run, logits, ref, ids, in_place=False, sample_ro
     # step 4
     src = logits.clone() if in_place else logits
     out = binding.PPOOutputs(src, in_place=in_place)
+    # every output starts as NaN: an element the kernels fail to write cannot pass for a zero
+    for t_ in (out.loss, out.dvalues, out.lp_new):
+        t_.fill_(float("nan"))
+    if not in_place:
+        out.dlogits.fill_(float("nan"))
     binding.ppo_loss_fwd_bwd(src, ids, lengths, _t(run.lp_old_in), _t(run.adv_in), _t(run.values_new_in),
                              _t(run.values_old_in), _t(run.ret_in), w.clip_eps, w.value_clip,
                              run.grad_scale, ws, out)
