@@ -75,6 +75,18 @@ const char* rlhf_status_string(int status);
 /* Text of the last CUDA runtime error this library saw on the calling thread ("" if none). */
 const char* rlhf_last_cuda_error(void);
 
+/* Host-side planning helper (no device access): which padded rows block `block` of a loss launch with
+ * `n_blocks` persistent blocks zero-fills, for a batch with n_valid valid and n_padded padded tokens.
+ * Valid rows are dealt round-robin (block i takes rows i, i+n_blocks, ...), so the first n_valid % n_blocks
+ * blocks hold one valid row more than the others; a valid row moves twice the bytes of a padded one (read +
+ * write against write only), so the other blocks first receive up to two padded rows each and the rest is
+ * dealt evenly.  The share is the contiguous range [*start, *start + *count) of the row-major list of padded
+ * tokens; the shares of blocks 0..n_blocks-1 tile [0, n_padded).  Returns RLHF_ERR_SHAPE for n_blocks <= 0,
+ * a block outside [0, n_blocks) or negative counts, RLHF_ERR_NULL for NULL outputs.  The loss kernels use
+ * the same rule on the device. */
+int rlhf_pad_share(long long n_valid, long long n_padded, int n_blocks, int block,
+                   long long* start, long long* count);
+
 /* Bytes of scratch that rlhf_gather_logprobs, rlhf_experience and rlhf_ppo_loss_fwd_bwd need for a batch of B x T
  * tokens: O(B*T), never O(B*T*V) -- at most 16*B*T + 65536.  0 if B or T is not positive.
  * The workspace must be 256-byte aligned and must have been cleared once with rlhf_workspace_init

@@ -25,6 +25,7 @@ _sz = ctypes.c_size_t
 SIGNATURES = {
     "rlhf_status_string": (ctypes.c_char_p, [_int]),
     "rlhf_last_cuda_error": (ctypes.c_char_p, []),
+    "rlhf_pad_share": (_int, [_i64, _i64, _int, _int, _vp, _vp]),
     "rlhf_workspace_bytes": (_sz, [_int, _int]),
     "rlhf_workspace_init": (_int, [_vp, _sz, _vp]),
     "rlhf_poll_status": (_int, [_vp, _vp]),
@@ -69,6 +70,14 @@ def lib() -> ctypes.CDLL:
             fn.argtypes = args
         _lib = handle
     return _lib
+
+
+def pad_share(n_valid: int, n_padded: int, n_blocks: int, block: int) -> Tuple[int, int]:
+    """(start, count) of the padded rows that `block` zero-fills in a loss launch (host-side helper)."""
+    start, count = _i64(0), _i64(0)
+    _check(lib().rlhf_pad_share(n_valid, n_padded, n_blocks, block, ctypes.byref(start), ctypes.byref(count)),
+           "rlhf_pad_share")
+    return int(start.value), int(count.value)
 
 
 def _check(status: int, where: str) -> None:

@@ -223,6 +223,16 @@ const char* rlhf_status_string(int status)
 
 const char* rlhf_last_cuda_error(void) { return g_cuda_error; }
 
+int rlhf_pad_share(long long n_valid, long long n_padded, int n_blocks, int block, long long* start, long long* count)
+{
+    if (!start || !count) return RLHF_ERR_NULL;
+    if (n_blocks <= 0 || block < 0 || block >= n_blocks || n_valid < 0 || n_padded < 0) return RLHF_ERR_SHAPE;
+    const PadShare s = pad_share(n_valid, n_padded, n_blocks, block);
+    *start = s.start;
+    *count = s.count;
+    return RLHF_OK;
+}
+
 size_t rlhf_workspace_bytes(int B, int T)
 {
     if (B <= 0 || T <= 0) return 0;

@@ -53,6 +53,21 @@ inline size_t dbuf_smem_bytes(unsigned row_bytes, bool any_alignment = false)
     return 2 * stride + kZeroBytes + 64;       // + 6 mbarriers
 }
 
+// Barrier over the NW consumer warps (named barrier 1) that also tells every thread whether `flag` was
+// set in any of them.
+template <int NW>
+__device__ __forceinline__ bool consumer_barrier_or(bool flag)
+{
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(any) : "r"((uint32_t)flag), "n"(NW * 32) : "memory");
+    return any != 0;
+}
+
 // Block-wide total of the partial sums, as consumer_reduce but with log2(NW) cross-warp steps.
 template <int NW>
 __device__ __forceinline__ Acc dbuf_reduce(const Acc& a, float2* s_part, const LabelInfo* s_lab, int warp, int lane)
@@ -94,10 +109,10 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     constexpr int kCons = NW * 32;
     constexpr int kThreads = kCons + 32;
     constexpr uint32_t kPiece = 16384;           // size of one bulk copy
-    constexpr uint32_t kStep = (uint32_t)kCons * 16u;       // bytes between a thread's consecutive vectors
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ long long s_cnt[33];
     __shared__ float2 s_part[2][32];
+    __shared__ __align__(16) float s_sum[2][NW];
     __shared__ LabelInfo s_lab[2];
     __shared__ RowInfo s_row[2];
     __shared__ double s_dbl[32];
@@ -276,8 +291,16 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         const uint4* src = (const uint4*)(smem + (size_t)buf * da.row_stride) + tid;
 
         // ---- pass 1: partition sum
+        // Every thread sums against the same reference exponent, taken from one vector of the row that all
+        // threads can see, so that the partial sums of the block add up without rescaling.  Blocks of 4 vectors
+        // are summed without range handling and their sums checked afterwards, once per row: a thread that met
+        // an entry 2^64 above the reference (or found no usable reference) redoes its share of the row with
+        // the careful routines under a reference of its own, and the block then merges by the general rule.
+        const float Mref = max8_scaled(((const uint4*)(smem + (size_t)buf * da.row_stride))[(kAny && eoff != 0) ? 1 : 0]);
         Acc a = acc_empty();
         float zy = 0.f;
+        bool redo = !(Mref > kFloorM);
+        a.M = Mref;
         auto sum_range = [&](int j0, int j1) {
             int j = j0;
             for (; j + 4 <= j1; j += 4) {
@@ -289,23 +312,48 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                     for (int u = 0; u < 4; ++u) add_special(a, q[u], j + u, zy);
                 } else {
                     const float vs = exp_sum_vecs<4>(q, -a.M);
-                    if (vs <= 1.8446744e19f) {
-                        a.s += vs;
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) acc_add_vec(a, q[u]);
-                    }
+                    a.s += vs;
+                    redo |= !(vs <= 1.8446744e19f);
                 }
             }
             for (; j < j1; ++j) add_special(a, src[(size_t)j * kCons], j, zy);
         };
-        if (cnt > 0 && jy != 0 && jfirst != 0 && jlast != 0) a.M = max8_scaled(src[0]);          // this thread's reference exponent for the row
         sum_range(0, head_cnt);
         mbar_wait(landed(buf, 1), use, p.status, aborted);
         sum_range(head_cnt, cnt);
+        if (redo) {
+            a = acc_empty();
+            zy = 0.f;
+            for (int j = 0; j < cnt; ++j) add_special(a, src[(size_t)j * kCons], j, zy);
+        }
+        const bool diverged = cnt > 0 && a.M != Mref;               // (a careful routine may also have raised the reference)
 
         if (owner) s_lab[par] = LabelInfo{zy, a.ey, a.M, 0.f};
-        const Acc tot = dbuf_reduce<NW>(a, s_part[par], &s_lab[par], warp, lane);
+        float ws = cnt > 0 ? a.s : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+        if (lane == 0) s_sum[par][warp] = ws;
+        Acc tot;
+        if (!consumer_barrier_or<NW>(diverged)) {
+            // common case: one reference for the whole block; every thread adds the warp sums in the same fixed tree
+            float v[NW];
+#pragma unroll
+            for (int w4 = 0; w4 < NW / 4; ++w4) {
+                const float4 t4 = ((const float4*)s_sum[par])[w4];
+                v[4 * w4] = t4.x; v[4 * w4 + 1] = t4.y; v[4 * w4 + 2] = t4.z; v[4 * w4 + 3] = t4.w;
+            }
+#pragma unroll
+            for (int st = 1; st < NW; st <<= 1)
+#pragma unroll
+                for (int w = 0; w + st < NW; w += 2 * st) v[w] += v[w + st];
+            tot.M = Mref;
+            tot.s = v[0];
+            tot.ey = s_lab[par].ey;
+        } else {
+            Acc mine = a;
+            if (cnt == 0) mine = acc_empty();
+            tot = dbuf_reduce<NW>(mine, s_part[par], &s_lab[par], warp, lane);
+        }
         const RowResult r = row_finish_fast(tot, s_lab[par].zy);
 
         float loss = 0.f, g = 0.f;

@@ -98,3 +98,34 @@ def test_binding_refuses_cpu_tensors():
     with pytest.raises(ValueError):
         binding.gather_logprobs(z, torch.zeros((1, 2), dtype=torch.int64), torch.ones(1, dtype=torch.int32),
                                 torch.zeros(8192, dtype=torch.uint8))
+
+
+@pytest.mark.parametrize("n_valid,n_padded,G", [(3006, 1090, 148), (0, 77, 148), (5, 0, 148), (148, 148, 148),
+                                                (9228, 7156, 148), (42800, 88272, 148), (7, 3, 4), (1000, 1, 148),
+                                                (149, 500, 148), (147, 293, 148)])
+def test_pad_share_tiles_the_padded_rows_and_balances_bytes(lib, n_valid, n_padded, G):
+    shares = [binding.pad_share(n_valid, n_padded, G, i) for i in range(G)]
+    # contiguous, in block order, covering [0, n_padded) exactly once
+    pos = 0
+    for start, count in shares:
+        assert start == pos and count >= 0
+        pos += count
+    assert pos == n_padded
+    # cost in units of one row written: a valid row counts 2 (read + write), a padded row 1
+    rows = [n_valid // G + (1 if i < n_valid % G else 0) for i in range(G)]
+    cost = [2 * r + c for r, (_, c) in zip(rows, shares)]
+    if n_padded >= 2 * (G - n_valid % G):
+        assert max(cost) - min(cost) <= 1               # enough padded rows to level the blocks
+    else:
+        # too few to level: they all go to the blocks with one valid row fewer, spread evenly
+        assert all(c == 0 for (_, c), r in zip(shares, rows) if r == max(rows) and max(rows) != min(rows))
+        lows = [c for (_, c), r in zip(shares, rows) if r == min(rows)]
+        assert max(lows) - min(lows) <= 1
+
+
+def test_pad_share_rejects_bad_arguments(lib):
+    s, c = ctypes.c_longlong(), ctypes.c_longlong()
+    assert lib.rlhf_pad_share(1, 1, 0, 0, ctypes.byref(s), ctypes.byref(c)) == 2
+    assert lib.rlhf_pad_share(1, 1, 4, 4, ctypes.byref(s), ctypes.byref(c)) == 2
+    assert lib.rlhf_pad_share(-1, 1, 4, 0, ctypes.byref(s), ctypes.byref(c)) == 2
+    assert lib.rlhf_pad_share(1, 1, 4, 0, None, ctypes.byref(c)) == 1
