@@ -47,51 +47,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
-// ---- 2^x without the special-function unit ------------------------------------------------------
-// ex2 runs at 16 results per clock per SM, and the row kernels need one per logit per pass, which is
-// what limits them once the memory side keeps up.  A fraction of the exponentials is therefore
-// evaluated on the FMA pipe, two at a time with the packed fp32x2 instructions of sm_100:
-//   x clamped to >= -127;  t = x + (1.5*2^23 + 127) rounds x to the nearest integer n and leaves n+127
-//   in the low mantissa bits of t;  f = x - n in [-1/2, 1/2];  2^f by a minimax polynomial;
-//   2^n = the bits of t shifted into the exponent field (n = -127 gives 0: results below 2^-126
-//   flush to zero like ex2.approx.ftz).
-// Maximum relative error of the polynomial: degree 4, 2.7e-6 (partition sums); degree 3, 7.5e-5
-// (gradients, which are rounded to bf16, half an ulp = 2e-3).
-constexpr float kPolyMagic = 12582912.f + 127.f;
-constexpr uint32_t kPolyMagicBits = 0x4B400000u;     // bits of 1.5*2^23; valid t: these bits + (n+127), n+127 in [0,254]
-
 __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
-
-// `seen` collects the bits of every t so that the caller can tell whether some x was >= 128
-// (see ex2_fma_in_range); pass-2 callers, whose x is bounded above, ignore it.
-template <int DEG>
-__device__ __forceinline__ float2 ex2_fma_pair(float2 x, uint32_t& seen)
-{
-    x.x = fmaxf(x.x, -127.f);
-    x.y = fmaxf(x.y, -127.f);
-    const float2 t = __fadd2_rn(x, splat2(kPolyMagic));
-    const float2 n = __fadd2_rn(t, splat2(-kPolyMagic));
-    const float2 f = __ffma2_rn(n, splat2(-1.f), x);
-    float2 p;
-    if (DEG == 3) {
-        p = __ffma2_rn(f, splat2(0.05517166852951050f), splat2(0.2426111251115799f));
-        p = __ffma2_rn(p, f, splat2(0.6932609677314758f));
-        p = __ffma2_rn(p, f, splat2(0.9999280571937561f));
-    } else {
-        p = __ffma2_rn(f, splat2(0.009570064023137093f), splat2(0.05591786280274391f));
-        p = __ffma2_rn(p, f, splat2(0.2402474582195282f));
-        p = __ffma2_rn(p, f, splat2(0.6931217908859253f));
-        p = __ffma2_rn(p, f, splat2(0.9999992847442627f));
-    }
-    const uint32_t tx = __float_as_uint(t.x), ty = __float_as_uint(t.y);
-    seen |= tx | ty;
-    return __fmul2_rn(p, make_float2(__uint_as_float(tx << 23), __uint_as_float(ty << 23)));
-}
-
-// True if every x given to ex2_fma_pair since `seen` was set to kPolyMagicBits was below 128, i.e. every
-// scale 2^n was representable.  (A larger x changes bits of t above the low eight; a smaller one cannot
-// occur after the clamp.)
-__device__ __forceinline__ bool ex2_fma_in_range(uint32_t seen) { return (seen & 0xffffff00u) == kPolyMagicBits; }
 
 __device__ __forceinline__ float2 unpack_bf16x2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
 

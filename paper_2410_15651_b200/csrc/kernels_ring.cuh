@@ -171,42 +171,25 @@ __device__ __forceinline__ float acc_add_vec_range(Acc& a, const uint4& q, int j
     return zy;
 }
 
-#ifndef RLHF_POLY_MASKS
-#define RLHF_POLY_MASKS 0x0, 0x0, 0x0
-#endif
-constexpr int kPolyMasks[3] = {RLHF_POLY_MASKS};
-constexpr int kSumPolyWords = kPolyMasks[0], kGradPolyEven = kPolyMasks[1], kGradPolyOdd = kPolyMasks[2];
-
-// dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.  kPolyWords: bit k set = entries 2k, 2k+1
-// take the FMA-pipe exponential (degree 3) instead of ex2.
-template <int kPolyWords>
-__device__ __forceinline__ uint4 grad_vec_mix(const uint4& q, float c2, uint32_t sign2)
+// dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.  The scaling runs two entries at a time on
+// the packed fp32x2 FMA of sm_100; the exponentials stay on the special-function unit.
+__device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sign2)
 {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
     uint32_t o[4];
-    uint32_t seen = 0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const float2 x = __ffma2_rn(unpack_bf16x2(w[k]), splat2(kLog2e), splat2(c2));
-        const float2 d = ((kPolyWords >> k) & 1) ? ex2_fma_pair<3>(x, seen) : make_float2(ex2(x.x), ex2(x.y));
-        o[k] = pack_bf16x2(d.x, d.y) ^ sign2;
+        o[k] = pack_bf16x2(ex2(x.x), ex2(x.y)) ^ sign2;
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// One vector on its own: a quarter of the entries on the FMA pipe.
-__device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sign2)
-{
-    return grad_vec_mix<kGradPolyEven>(q, c2, sign2);
-}
-
-// U vectors: 3 of every 8 exponentials on the FMA pipe (1 word of even vectors, 2 of odd ones), the
-// mix at which the special-function unit and the issue slots are about equally loaded.
 template <int U>
 __device__ __forceinline__ void grad_vecs(const uint4 (&q)[U], uint4 (&o)[U], float c2, uint32_t sign2)
 {
 #pragma unroll
-    for (int u = 0; u < U; ++u) o[u] = (u & 1) ? grad_vec_mix<kGradPolyOdd>(q[u], c2, sign2) : grad_vec_mix<kGradPolyEven>(q[u], c2, sign2);
+    for (int u = 0; u < U; ++u) o[u] = grad_vec(q[u], c2, sign2);
 }
 
 __device__ __forceinline__ void patch_label(uint4& o, int j, float value)
@@ -262,27 +245,22 @@ __device__ __forceinline__ Acc consumer_reduce(const Acc& a, float2* s_part, con
 }
 
 // ---------------------------------------------------------------- the kernel
-// Sum of the exponentials of U vectors against one reference exponent.  A quarter of them (the last
-// word of every vector) is evaluated on the FMA pipe (degree 4).  No range handling: if an entry is 2^128
-// or more above the reference the result is +inf, and the caller, which redoes any block whose sum
-// exceeds 2^64, takes the careful path.
+// Sum of the exponentials of U vectors against one reference exponent (no range check): scaling and
+// accumulation two entries at a time (packed fp32x2), one ex2 per entry.
 template <int U>
 __device__ __forceinline__ float exp_sum_vecs(const uint4 (&q)[U], float negM)
 {
     float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-    uint32_t seen = kPolyMagicBits;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const float2 x = __ffma2_rn(unpack_bf16x2(w[k]), splat2(kLog2e), splat2(negM));
-            const float2 e = ((kSumPolyWords >> k) & 1) ? ex2_fma_pair<4>(x, seen) : make_float2(ex2(x.x), ex2(x.y));
-            acc[k & 1] = __fadd2_rn(acc[k & 1], e);
+            acc[k & 1] = __fadd2_rn(acc[k & 1], make_float2(ex2(x.x), ex2(x.y)));
         }
     }
-    const float vs = (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
-    return ex2_fma_in_range(seen) ? vs : __int_as_float(0x7f800000);
+    return (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
 }
 
 __device__ __forceinline__ float max8_scaled(const uint4& q)
