@@ -551,7 +551,7 @@ inline RingPlan plan_ring(unsigned row_bytes, int sm_smem, int block_smem_max)
     // rows larger than shared memory are streamed twice.  One block of 16 consumer warps per SM
     // keeps the number of rows in flight at the number of SMs, so that the second read of a row
     // (a few tens of microseconds after the first) is still served by L2.
-    const int NW = 16, U = 2;
+    const int NW = 16, U = 4;
     const size_t chunk = (size_t)NW * 32 * 16 * U;
     const int chunks = (int)((row_bytes + chunk - 1) / chunk);
     int S = 2;
