@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch of the loss kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
 # ncu capture summarised under profiles/, valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"sources_sha256": "053beca621276d5d", "workload": "opt", "bytes_per_launch": 656014592}
+NCU_TRAFFIC = {"sources_sha256": "8ac75a4d50aa59bb", "workload": "opt", "bytes_per_launch": 654396928}
 
 
 def sources_digest() -> str:
