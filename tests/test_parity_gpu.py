@@ -310,6 +310,34 @@ def test_rows_larger_than_shared_memory(oracle, V, in_place):
         dlogits_properties(run, out, batch["ids"], batch["actor"])
 
 
+@pytest.mark.parametrize("V,in_place", [(32000, False), (50272, True), (4096, False)])
+def test_rows_that_leave_the_common_reference_exponent(oracle, V, in_place):
+    # The loss kernel for rows of 16-111 KB sums a row against one reference exponent taken from the row's first
+    # 8 logits and falls back to per-thread references when that does not hold.  Rows built to force every branch:
+    # first 8 logits all -inf (no reference); first 8 logits far below the rest (entries > 2^64 above the
+    # reference: spikes of +60..+90, at the label and elsewhere); first 8 logits far above the rest (everything else
+    # more than 100 binades below the reference); -inf inside the first vector only.  V=4096 takes the chunk-ring kernel.
+    w = inputs.scaled(inputs.WORKLOADS["llama2"], V=V, B=2, T=6, lengths="uniform:6:6", seed=90 + V % 11)
+    batch = inputs.make_batch(w, device=DEV)
+    a = batch["actor"]
+    a[0, 0, :8] = float("-inf")
+    a[0, 1, 1234] = 80.0                              # spike elsewhere
+    a[0, 2, int(batch["ids"][0, 2])] = 90.0           # spike at the label
+    a[0, 3, :8] = 70.0                                # reference far above the rest of the row
+    a[0, 4, 1:5] = float("-inf")
+    a[0, 5, :8] = -60.0                               # reference far below: every other entry is ~2^86 above it
+    a[1, 0, V - 1] = 75.0
+    a[1, 1, :16] = float("-inf")
+    for b_, t_ in ((0, 0), (0, 4), (1, 1)):           # the label must not sit on a deleted entry
+        if int(batch["ids"][b_, t_]) < 16:
+            batch["ids"][b_, t_] = 100
+    batch["ref"] = a.clone()
+    run = OracleRun(oracle, w, batch)
+    out, _ = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], in_place=in_place, all_rows=True)
+    if not in_place:
+        dlogits_properties(run, out, batch["ids"], batch["actor"])
+
+
 def test_gpt2_vocabulary_rows_off_16_byte_boundaries(oracle):
     # V = 50257: every row starts 2 bytes further off a 16-byte boundary than the one before it
     w = inputs.scaled(inputs.WORKLOADS["gpt2"], B=3, T=12, lengths="uniform:5:12")
