@@ -53,21 +53,6 @@ inline size_t dbuf_smem_bytes(unsigned row_bytes, bool any_alignment = false)
     return 2 * stride + kZeroBytes + 64;       // + 6 mbarriers
 }
 
-// Barrier over the NW consumer warps (named barrier 1) that also tells every thread whether `flag` was
-// set in any of them.
-template <int NW>
-__device__ __forceinline__ bool consumer_barrier_or(bool flag)
-{
-    uint32_t any;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, %2, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(any) : "r"((uint32_t)flag), "n"(NW * 32) : "memory");
-    return any != 0;
-}
-
 // Block-wide total of the partial sums, as consumer_reduce but with log2(NW) cross-warp steps.
 template <int NW>
 __device__ __forceinline__ Acc dbuf_reduce(const Acc& a, float2* s_part, const LabelInfo* s_lab, int warp, int lane)
@@ -336,18 +321,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         Acc tot;
         if (!consumer_barrier_or<NW>(diverged)) {
             // common case: one reference for the whole block; every thread adds the warp sums in the same fixed tree
-            float v[NW];
-#pragma unroll
-            for (int w4 = 0; w4 < NW / 4; ++w4) {
-                const float4 t4 = ((const float4*)s_sum[par])[w4];
-                v[4 * w4] = t4.x; v[4 * w4 + 1] = t4.y; v[4 * w4 + 2] = t4.z; v[4 * w4 + 3] = t4.w;
-            }
-#pragma unroll
-            for (int st = 1; st < NW; st <<= 1)
-#pragma unroll
-                for (int w = 0; w + st < NW; w += 2 * st) v[w] += v[w + st];
             tot.M = Mref;
-            tot.s = v[0];
+            tot.s = sum_warp_sums<NW>(s_sum[par]);
             tot.ey = s_lab[par].ey;
         } else {
             Acc mine = a;

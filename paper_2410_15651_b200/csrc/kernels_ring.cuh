@@ -244,6 +244,38 @@ __device__ __forceinline__ Acc consumer_reduce(const Acc& a, float2* s_part, con
     return tot;
 }
 
+// Barrier over the NW consumer warps (named barrier 1) that also tells every thread whether `flag` was
+// set in any of them.
+template <int NW>
+__device__ __forceinline__ bool consumer_barrier_or(bool flag)
+{
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(any) : "r"((uint32_t)flag), "n"(NW * 32) : "memory");
+    return any != 0;
+}
+
+// Sum of the NW warp sums published in `s_sum` (16-byte aligned), added by every thread in the same fixed tree.
+template <int NW>
+__device__ __forceinline__ float sum_warp_sums(const float* s_sum)
+{
+    float v[NW];
+#pragma unroll
+    for (int w4 = 0; w4 < NW / 4; ++w4) {
+        const float4 t4 = ((const float4*)s_sum)[w4];
+        v[4 * w4] = t4.x; v[4 * w4 + 1] = t4.y; v[4 * w4 + 2] = t4.z; v[4 * w4 + 3] = t4.w;
+    }
+#pragma unroll
+    for (int st = 1; st < NW; st <<= 1)
+#pragma unroll
+        for (int w = 0; w + st < NW; w += 2 * st) v[w] += v[w + st];
+    return v[0];
+}
+
 // ---------------------------------------------------------------- the kernel
 // Sum of the exponentials of U vectors against one reference exponent (no range check): scaling and
 // accumulation two entries at a time (packed fp32x2), one ex2 per entry.
@@ -283,6 +315,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ long long s_cnt[33];
     __shared__ float2 s_part[2][32];
+    __shared__ __align__(16) float s_sum[2][NW];
     __shared__ LabelInfo s_lab[2];
     __shared__ double s_dbl[32];
 
@@ -398,18 +431,24 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
         const uint32_t phase0 = phase;
 
         // ---- pass 1: partition sum
+        // Every thread starts from the same reference exponent (the scaled maximum of the row's first vector), so
+        // that the block's partial sums add up without rescaling unless some thread had to raise its reference.
         Acc a = acc_empty();
         float zy = 0.f;
+        float Mref = kFloorM;
         const bool owner = (yvec % kCons) == (uint32_t)tid;      // this thread sums the generated token's vector
         for (int c = 0; c < chunks; ++c) {
             mbar_wait(full_addr + 8u * slot, phase, p.status, aborted);
             const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk) + tid;
+            if (c == 0) {
+                Mref = max8_scaled(*(const uint4*)(smem + (size_t)slot * kChunk));
+                if (Mref > kFloorM) a.M = Mref;
+            }
             if (c < full_chunks && c != ychunk) {
                 // common case: every vector exists and none holds the generated token
                 uint4 q[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) q[u] = src[u * kCons];
-                if (c == 0) a.M = max8_scaled(q[0]);               // thread's reference exponent for this row
                 const float vs = exp_sum_vecs<U>(q, -a.M);
                 if (vs <= 1.8446744e19f) {
                     a.s += vs;
@@ -437,7 +476,18 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
             if (++slot == S) { slot = 0; phase ^= 1u; }
         }
         if (owner) s_lab[par] = LabelInfo{zy, a.ey, a.M, 0.f};
-        const Acc tot = consumer_reduce<NW>(a, s_part[par], &s_lab[par], warp, lane);
+        float ws = a.s;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, o);
+        if (lane == 0) s_sum[par][warp] = ws;
+        Acc tot;
+        if (!consumer_barrier_or<NW>(a.M != Mref)) {
+            tot.M = Mref;
+            tot.s = sum_warp_sums<NW>(s_sum[par]);
+            tot.ey = s_lab[par].ey;
+        } else {
+            tot = consumer_reduce<NW>(a, s_part[par], &s_lab[par], warp, lane);
+        }
         const RowResult r = row_finish(tot, s_lab[par].zy);
 
         // scalars of the next row, in flight while this row is finished
