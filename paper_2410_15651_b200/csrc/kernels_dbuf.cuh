@@ -267,11 +267,15 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         const bool owner = (yvec % kCons) == (uint32_t)tid;
         const int jy = owner ? (int)(yvec / kCons) : -1;            // which of this thread's vectors holds the label
         // one vector of this thread, with whatever is special about it
+        // (kAny) the first and last vector of the row, foreign entries turned into -inf; any other vector unchanged
+        auto in_row = [&](const uint4& q, int j) {
+            if (kAny && j == jfirst) return mask_vec_outside(q, (int)eoff, 8);
+            if (kAny && j == jlast) return mask_vec_outside(q, 0, (int)((eoff + (uint32_t)p.V) & 7u));
+            return q;
+        };
         auto add_special = [&](Acc& acc, const uint4& q, int j, float& zy_out) {
-            if (kAny && j == jfirst) zy_out += acc_add_vec_range(acc, q, (int)eoff, 8, j == jy ? yj : -1);
-            else if (kAny && j == jlast) zy_out += acc_add_vec_range(acc, q, 0, (int)((eoff + (uint32_t)p.V) & 7u), j == jy ? yj : -1);
-            else if (j == jy) zy_out = acc_add_vec_label(acc, q, yj);
-            else acc_add_vec(acc, q);
+            if (j == jy) zy_out = acc_add_vec_label(acc, in_row(q, j), yj);
+            else acc_add_vec(acc, in_row(q, j));
         };
         const uint4* src = (const uint4*)(smem + (size_t)buf * da.row_stride) + tid;
 
@@ -292,9 +296,16 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 uint4 q[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) q[u] = src[(size_t)(j + u) * kCons];
-                if ((unsigned)(jy - j) < 4u || (kAny && ((unsigned)(jfirst - j) < 4u || (unsigned)(jlast - j) < 4u))) {
+                if (kAny && ((unsigned)(jfirst - j) < 4u || (unsigned)(jlast - j) < 4u)) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) add_special(a, q[u], j + u, zy);
+                    for (int u = 0; u < 4; ++u) q[u] = in_row(q[u], j + u);
+                }
+                if ((unsigned)(jy - j) < 4u) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (j + u == jy) zy = acc_add_vec_label(a, q[u], yj);
+                        else acc_add_vec(a, q[u]);
+                    }
                 } else {
                     const float vs = exp_sum_vecs<4>(q, -a.M);
                     a.s += vs;

@@ -171,6 +171,19 @@ __device__ __forceinline__ float acc_add_vec_range(Acc& a, const uint4& q, int j
     return zy;
 }
 
+// Entries of a vector outside [jlo, jhi) replaced by -inf (bf16 0xFF80): they then add nothing to a partition sum.
+// For the first or last vector of a row that does not start or end on a 16-byte boundary.
+__device__ __forceinline__ uint4 mask_vec_outside(const uint4& q, int jlo, int jhi)
+{
+    uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (i < jlo || i >= jhi)
+            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | 0xff800000u) : ((w[i >> 1] & 0xffff0000u) | 0x0000ff80u);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.  The scaling runs two entries at a time on
 // the packed fp32x2 FMA of sm_100; the exponentials stay on the special-function unit.
 __device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sign2)
