@@ -112,7 +112,7 @@ def visible_gpu_index(local_rank: int) -> int:
 class Path:
     """All buffers of one step, resident on the device, and the step itself (C-ABI calls only)."""
 
-    def __init__(self, w, batch, dev, fused=True):
+    def __init__(self, w, batch, dev, fused=True, in_place=False):
         import torch
         from paper_2410_15651_b200 import binding
         self.b, self.w, self.binding = batch, w, binding
@@ -124,7 +124,11 @@ class Path:
         self.exp.lp_actor, self.exp.lp_ref, self.exp.rewards = self.lp_act, self.lp_ref, self.rewards
         self.exp.adv, self.exp.returns = self.adv, self.ret
         self.fused = fused
-        self.out = binding.PPOOutputs(batch["actor"])
+        # in place: the gradient overwrites the logits it was computed from.  The loss call then gets a copy of
+        # the actor logits of its own, so that the experience phase of the next step still reads logits; after
+        # the first step that copy holds gradients, which costs the same traffic to read.
+        self.loss_logits = batch["actor"].clone() if in_place else batch["actor"]
+        self.out = binding.PPOOutputs(self.loss_logits, in_place=in_place)
         self.N = int(batch["lengths"].sum().item())
         # old-policy log-probs = current + N(0, sigma^2) on valid tokens, prepared once outside the timed region
         cur = binding.gather_logprobs(batch["actor"], batch["ids"], batch["lengths"], self.ws)
@@ -142,7 +146,7 @@ class Path:
             self._experience_separate()
         if ev is not None:
             ev[0].record()
-        k.ppo_loss_fwd_bwd(b["actor"], b["ids"], b["lengths"], self.lp_old, self.adv, b["values_new"],
+        k.ppo_loss_fwd_bwd(self.loss_logits, b["ids"], b["lengths"], self.lp_old, self.adv, b["values_new"],
                            b["values_old"], self.ret, w.clip_eps, w.value_clip, float(self.N), self.ws, self.out)
         if ev is not None:
             ev[1].record()
@@ -177,7 +181,7 @@ def run_ours(args):
     if args.sequences > 0:
         w = inputs.scaled(w, B=args.sequences)
     batch = inputs.make_batch(w, device=dev)
-    path = Path(w, batch, dev, fused=not args.separate_calls)
+    path = Path(w, batch, dev, fused=not args.separate_calls, in_place=args.in_place)
     B, T, V = w.B, w.T, w.V
     n_valid = path.N
 
@@ -197,6 +201,7 @@ def run_ours(args):
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(visible_gpu_index(local_rank))
     sync_all()
+    mem_before = (torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev))
     sampler.start()
     t0.record()
     for i in range(K):
@@ -204,6 +209,7 @@ def run_ours(args):
     t1.record()
     sync_all()
     clocks = sampler.stop()
+    mem_after = (torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev))
     elapsed_ms = t0.elapsed_time(t1)
     loss_ms = sum(a.elapsed_time(b) for a, b in inner) / K
     assert binding.poll_status(path.ws) == 0
@@ -260,6 +266,10 @@ def run_ours(args):
         "config": {"workload": f"{args.workload}: B={B} T={T} V={V} bf16 logits, {n_valid} response tokens per GPU",
                    "l2": "inputs larger than L2 (%.2f GB touched per step)" % (step_bytes / 1e9 + 0.0),
                    "multi_gpu": "independent batch per rank, no data-path collective",
+                   "dlogits": "in place (over a copy of the logits)" if args.in_place else "separate bf16 [B,T,V] buffer",
+                   "workspace_bytes": int(path.ws.numel()), "workspace_bound_16BT_plus_64K": 16 * B * T + 65536,
+                   "torch_allocated_bytes_before_after": [mem_before[0], mem_after[0]],
+                   "torch_reserved_bytes_before_after": [mem_before[1], mem_after[1]],
                    "calls_per_step": ("rlhf_gather_logprobs x2, rlhf_kl_reward, rlhf_gae, rlhf_ppo_loss_fwd_bwd"
                                       if args.separate_calls else "rlhf_experience, rlhf_ppo_loss_fwd_bwd")},
         "clocks": clocks, "gpu_launches": path.launches_per_step * K,
@@ -375,6 +385,7 @@ def main():
     ap.add_argument("--sequences", type=int, default=0,
                     help="override the number of sequences B of the workload (smaller cases for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--in-place", action="store_true", help="dlogits overwrite the logits given to the loss call")
     ap.add_argument("--separate-calls", action="store_true",
                     help="experience phase as four calls (2 x gather_logprobs, kl_reward, gae) instead of rlhf_experience")
     args = ap.parse_args()
