@@ -1,5 +1,6 @@
 """CUDA path against the CPU oracle at the full sizes of the OPT-shaped, Llama-2-shaped,
-large-vocabulary and ragged workloads, in the launch configuration the benchmark times.
+large-vocabulary, ragged and GPT-2-shaped (rows off 16-byte boundaries) workloads, in the launch
+configuration the benchmark times.
 
 Every O(B*T) output (log-probs of all rows for actor and reference, rewards, advantages, returns,
 dvalues, both losses) is compared in full: the oracle computes all of them.  The bf16 logits
@@ -19,7 +20,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("name,in_place", [("opt", False), ("opt", True), ("llama2", False),
-                                           ("large_vocab", False), ("ragged", False)])
+                                           ("large_vocab", False), ("ragged", False), ("gpt2", False), ("gpt2", True)])
 def test_full_size(oracle, name, in_place):
     w = inputs.WORKLOADS[name]
     batch = inputs.make_batch(w, device=DEV)
