@@ -52,50 +52,91 @@ def hbm_peak():
 
 
 class ClockSampler:
-    """Samples SM clock, power and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    """Samples SM clock, power and clock-event reasons of one GPU while a region runs (read-only queries):
+    through NVML in a thread of this process every 20 ms, or, where the NVML module is missing, through an
+    nvidia-smi child process every 100 ms."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+    MASKS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
     def __init__(self, index: int):
         self.index = index
         self.proc = None
         self.out = None
+        self.thread = None
+        self.rows = []          # (sm_mhz, sm_max_mhz, watts, set of active reasons)
+        self.how = None
+
+    def _nvml_loop(self, nvml, handle):
+        import threading
+        self._stop = threading.Event()
+
+        def loop():
+            mx = nvml.nvmlDeviceGetMaxClockInfo(handle, nvml.NVML_CLOCK_SM)
+            while True:
+                try:
+                    try:
+                        mask = nvml.nvmlDeviceGetCurrentClocksEventReasons(handle)
+                    except AttributeError:
+                        mask = nvml.nvmlDeviceGetCurrentClocksThrottleReasons(handle)
+                    self.rows.append((float(nvml.nvmlDeviceGetClockInfo(handle, nvml.NVML_CLOCK_SM)), float(mx),
+                                      nvml.nvmlDeviceGetPowerUsage(handle) / 1000.0,
+                                      {n for n, m in self.MASKS.items() if mask & m}))
+                except Exception:
+                    pass
+                if self._stop.wait(0.02):
+                    return
+
+        self.thread = threading.Thread(target=loop, daemon=True)
+        self.thread.start()
 
     def start(self):
+        try:
+            import pynvml as nvml
+            nvml.nvmlInit()
+            self._nvml_loop(nvml, nvml.nvmlDeviceGetHandleByIndex(self.index))
+            self.how = "nvml, 20 ms"
+            return
+        except Exception:
+            self.thread = None
         try:
             self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                  "-i", str(self.index), "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+            self.how = "nvidia-smi, 100 ms"
         except Exception:
             self.proc = None
 
     def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        self.out.flush()
-        rows = [l.strip().split(", ") for l in open(self.out.name) if l.strip()]
-        os.unlink(self.out.name)
-        sm, mx, pw, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+        elif self.proc is not None:
+            self.proc.terminate()
             try:
-                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+                self.proc.wait(timeout=5)
             except Exception:
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.strip().lower() == "active":
-                    reasons.add(n)
-        sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+                self.proc.kill()
+            self.out.flush()
+            for l in open(self.out.name):
+                r = l.strip().split(", ")
+                try:
+                    self.rows.append((float(r[0]), float(r[1]), float(r[2]),
+                                      {n for n, v in zip(self.NAMES, r[3:7]) if v.strip().lower() == "active"}))
+                except Exception:
+                    continue
+            os.unlink(self.out.name)
+        else:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML module and no nvidia-smi"]}
+        sm = sorted(r[0] for r in self.rows)
+        reasons = set().union(*[r[3] for r in self.rows]) if self.rows else set()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max((r[1] for r in self.rows), default=None),
+                "power_w_max": max((r[2] for r in self.rows), default=None), "samples": len(sm),
+                "reasons": sorted(reasons), "sampled_by": self.how}
 
 
 def visible_gpu_index(local_rank: int) -> int:
