@@ -68,6 +68,17 @@ def _load():
         lib.oracle_ppo_loss.restype = None
         lib.oracle_ppo_loss.argtypes = [_vp] * 7 + [ctypes.c_int, ctypes.c_int, _dbl, _dbl, _dbl,
                                                     _vp, _vp, _vp, _vp]
+        lib.oracle_f16_to_double.restype = _dbl
+        lib.oracle_f16_to_double.argtypes = [ctypes.c_uint16]
+        lib.oracle_round_f16.restype = _dbl
+        lib.oracle_round_f16.argtypes = [_dbl]
+        lib.oracle_token_entropy.restype = None
+        lib.oracle_token_entropy.argtypes = [_vp, ctypes.c_int, _i64, _i64, _vp, ctypes.c_int, ctypes.c_int,
+                                             _i64, _vp]
+        lib.oracle_ppo_stats.restype = None
+        lib.oracle_ppo_stats.argtypes = [_vp, _vp, _vp, _vp, ctypes.c_int, ctypes.c_int, _dbl, _vp, _vp]
+        lib.oracle_whiten.restype = None
+        lib.oracle_whiten.argtypes = [_vp, _vp, ctypes.c_int, ctypes.c_int, _dbl, _vp]
         lib.oracle_dlogits_rows.restype = None
         lib.oracle_dlogits_rows.argtypes = [_vp, ctypes.c_int, _i64, _i64, _vp, _i64, _vp,
                                             ctypes.c_int, ctypes.c_int, _i64, _vp, _vp, _i64, _vp]
@@ -95,15 +106,18 @@ def _f64(a, shape=None) -> np.ndarray:
 
 
 def _logits_view(logits: np.ndarray):
-    """Return (array kept alive, is_bf16, stride_b, stride_t) for a [B,T,V] uint16 or float64 array
-    whose last axis is contiguous; the first two axes may be strided (a view of a longer tensor)."""
+    """Return (element type code, stride_b, stride_t) for a [B,T,V] array whose last axis is contiguous; the
+    first two axes may be strided (a view of a longer tensor).  uint16 = bf16 bit patterns (code 1),
+    float16 = IEEE binary16 (code 2, its bit patterns are passed), float64 (code 0)."""
     assert logits.ndim == 3
     if logits.dtype == np.uint16:
         is_bf16 = 1
+    elif logits.dtype == np.float16:
+        is_bf16 = 2
     elif logits.dtype == np.float64:
         is_bf16 = 0
     else:
-        raise TypeError("logits must be uint16 (bf16 bit patterns) or float64")
+        raise TypeError("logits must be uint16 (bf16 bit patterns), float16 or float64")
     item = logits.dtype.itemsize
     if logits.shape[2] > 1 and logits.strides[2] != item:
         raise ValueError("vocabulary axis must be contiguous")
@@ -138,6 +152,29 @@ def bf16_ulp(x) -> np.ndarray:
         lg = np.floor(np.log2(np.where(x > 0, x, 1.0)))
     lg = np.maximum(lg, -126.0)
     return np.where(x > 0, np.exp2(lg - 7.0), 2.0 ** -133)
+
+
+def f16_to_double(bits) -> np.ndarray:
+    """Exact widening of IEEE binary16 bit patterns (uint16) to float64."""
+    lib = _load()
+    bits = np.asarray(bits, dtype=np.uint16)
+    return np.vectorize(lambda h: lib.oracle_f16_to_double(int(h)), otypes=[np.float64])(bits)
+
+
+def round_f16(x) -> np.ndarray:
+    """Round float64 values to the nearest binary16 (ties to even); returned as float64."""
+    lib = _load()
+    x = np.asarray(x, dtype=np.float64)
+    return np.vectorize(lambda v: lib.oracle_round_f16(float(v)), otypes=[np.float64])(x)
+
+
+def f16_ulp(x) -> np.ndarray:
+    """Spacing of binary16 numbers at |x|: 2^(floor(log2|x|) - 10), with the subnormal floor 2^-24."""
+    x = np.abs(np.asarray(x, dtype=np.float64))
+    with np.errstate(divide="ignore"):
+        lg = np.floor(np.log2(np.where(x > 0, x, 1.0)))
+    lg = np.maximum(lg, -14.0)
+    return np.where(x > 0, np.exp2(lg - 10.0), 2.0 ** -24)
 
 
 def row_lse(z) -> float:
@@ -235,4 +272,38 @@ def dlogits_rows(logits, ids, lengths, g, rows) -> np.ndarray:
     out = np.empty((rows.size, V), dtype=np.float64)
     _load().oracle_dlogits_rows(_p(logits), is_bf16, sb, st, _p(ids), isb, _p(lengths),
                                 B, T, V, _p(g), _p(rows), rows.size, _p(out))
+    return out
+
+
+def token_entropy(logits: np.ndarray, lengths) -> np.ndarray:
+    """Entropy (nats) of the softmax of every valid row, float64 [B,T]; 0 at padded positions."""
+    B, T, V = logits.shape
+    dtype, sb, st = _logits_view(logits)
+    lengths = _lengths(lengths, B)
+    out = np.empty((B, T), dtype=np.float64)
+    _load().oracle_token_entropy(_p(logits), dtype, sb, st, _p(lengths), B, T, V, _p(out))
+    return out
+
+
+def ppo_stats(lp_new, lp_old, adv, lengths, clip_eps: float):
+    """(approx_kl, clip_frac) over the valid tokens: mean of rho - 1 - log rho, and the share of tokens
+    whose gradient the clip switches off."""
+    lp_new = _f64(lp_new)
+    B, T = lp_new.shape
+    lp_old, adv = _f64(lp_old, (B, T)), _f64(adv, (B, T))
+    lengths = _lengths(lengths, B)
+    kl, cf = _dbl(0.0), _dbl(0.0)
+    _load().oracle_ppo_stats(_p(lp_new), _p(lp_old), _p(adv), _p(lengths), B, T, float(clip_eps),
+                             ctypes.byref(kl), ctypes.byref(cf))
+    return kl.value, cf.value
+
+
+def whiten(adv, lengths, eps: float = 1e-8) -> np.ndarray:
+    """Advantages whitened over the valid tokens of the batch: (A - mean) / sqrt(var + eps), population
+    variance; 0 at padded positions."""
+    adv = _f64(adv)
+    B, T = adv.shape
+    lengths = _lengths(lengths, B)
+    out = np.empty((B, T), dtype=np.float64)
+    _load().oracle_whiten(_p(adv), _p(lengths), B, T, float(eps), _p(out))
     return out

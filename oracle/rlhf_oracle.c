@@ -26,7 +26,7 @@
  *      is added at the last valid token t = len-1; nothing is added if len = 0.
  *  R3  GAE: the value after the last valid token is 0; there is no T+1-th value.
  *  R4  padded positions (t >= len) are ignored on input and produce 0 on every output.
- *  R5  no advantage whitening.
+ *  R5  no advantage whitening unless the caller asks for it (then R16).
  *  R6  both losses are token means over the whole batch: divided by N = sum_b len_b;
  *      if N = 0 both losses and every gradient are 0.
  *  R7  policy loss per token  l = max(-A*rho, -A*clip(rho, 1-eps, 1+eps)),  rho = exp(lp_new - lp_old);
@@ -37,7 +37,17 @@
  *  R10 grad_scale multiplies every gradient (it is the upstream dL).
  *  R11 a logit of -inf is a deleted vocabulary entry: it adds 0 to the partition sum and gets
  *      gradient 0.  It must not sit at the label, and a row must keep one finite logit.
- *  R12 bf16 logits are widened exactly; bf16 output rounding is round-to-nearest-even.
+ *  R12 bf16 logits are widened exactly; bf16 output rounding is round-to-nearest-even.  The same holds
+ *      for IEEE binary16 (fp16) logits, the other 16-bit type the paper's model families are run in.
+ *  R13 token entropy (a monitor of the policy, not a loss term: R9) is the Shannon entropy of the
+ *      softmax in nats, H = -sum_v p_v log p_v; deleted entries (R11) add 0.
+ *  R14 the policy-deviation monitor ("approximate KL") is the non-negative estimator
+ *      mean over valid tokens of (rho - 1) - log rho,  rho = exp(lp_new - lp_old).
+ *  R15 the clip fraction is the share of valid tokens whose gradient the clip switches off, i.e.
+ *      whose clipped term is strictly larger than the unclipped one (the complement of R7's branch).
+ *  R16 advantage whitening (optional, between GAE and the loss; off unless asked for, R5):
+ *      (A - mean) / sqrt(var + eps) over the valid tokens of the whole batch, var the population
+ *      variance (divided by N); padded positions give 0; N = 0 gives all zeros.
  *
  * Layout: every [B,T] array is row-major with T contiguous.  Logits are addressed as
  * base[b*stride_b + t*stride_t + v] (strides in elements), ids as ids[b*ids_stride_b + t].
@@ -94,6 +104,34 @@ double oracle_round_bf16(double x)
     return r;
 }
 
+/* exact widening of one IEEE binary16 bit pattern (R12): 1 sign, 5 exponent (bias 15), 10 fraction bits */
+static double f16_to_double(uint16_t h)
+{
+    int sign = (h >> 15) & 1, ex = (h >> 10) & 0x1f, fr = h & 0x3ff;
+    double v;
+    if (ex == 0) v = ldexp((double)fr, -24);                    /* zero and subnormals: fr * 2^-24 */
+    else if (ex == 31) v = fr ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)fr / 1024.0, ex - 15);
+    return sign ? -v : v;
+}
+
+double oracle_f16_to_double(uint16_t h) { return f16_to_double(h); }
+
+/* Round a double to the nearest binary16 value, ties to even (R12); returned as a double.
+ * binary16 has 11 significant bits, smallest normal 2^-14, subnormal spacing 2^-24, largest 65504. */
+double oracle_round_f16(double x)
+{
+    if (isnan(x) || isinf(x) || x == 0.0) return x;
+    int e;
+    (void)frexp(fabs(x), &e);
+    int lg = e - 1;
+    if (lg < -14) lg = -14;
+    double ulp = ldexp(1.0, lg - 10);
+    double r = nearbyint(x / ulp) * ulp;
+    if (fabs(r) >= 65536.0) return x > 0 ? INFINITY : -INFINITY;
+    return r;
+}
+
 /* log sum_v exp(z_v), two passes: max, then sum of exp(z - max).  -inf entries add 0 (R11). */
 static double row_lse(const double* z, i64 V)
 {
@@ -109,13 +147,15 @@ static double row_lse(const double* z, i64 V)
 
 double oracle_row_lse_f64(const double* z, i64 V) { return row_lse(z, V); }
 
-static void widen_row(const uint16_t* src, i64 V, double* dst)
+/* element type of a logits tensor: 0 = float64, 1 = bf16 bit patterns, 2 = binary16 bit patterns */
+static void widen_row(const uint16_t* src, i64 V, double* dst, int dtype)
 {
-    for (i64 v = 0; v < V; ++v) dst[v] = bf16_to_double(src[v]);
+    if (dtype == 2) for (i64 v = 0; v < V; ++v) dst[v] = f16_to_double(src[v]);
+    else for (i64 v = 0; v < V; ++v) dst[v] = bf16_to_double(src[v]);
 }
 
 /* Step 1: lp[b,t] = z[b,t,y] - log sum_v exp z[b,t,v] for t < len_b, 0 elsewhere (R4).
- * `is_bf16` selects the element type of `logits` (uint16 bit patterns or double).
+ * `is_bf16` selects the element type of `logits`: 0 = double, 1 = bf16 bit patterns, 2 = binary16 bit patterns.
  * Returns 0, or 1 if some id or length was out of range (that token is given lp = NaN). */
 int oracle_gather_logprobs(const void* logits, int is_bf16, i64 stride_b, i64 stride_t,
                            const i64* ids, i64 ids_stride_b, const int32_t* lengths,
@@ -146,7 +186,7 @@ int oracle_gather_logprobs(const void* logits, int is_bf16, i64 stride_b, i64 st
             }
             i64 off = (i64)b * stride_b + (i64)t * stride_t;
             const double* zr;
-            if (is_bf16) { widen_row((const uint16_t*)logits + off, V, z); zr = z; }
+            if (is_bf16) { widen_row((const uint16_t*)logits + off, V, z, is_bf16); zr = z; }
             else zr = (const double*)logits + off;
             out_lp[r] = zr[y] - row_lse(zr, V);
         }
@@ -270,7 +310,7 @@ void oracle_dlogits_rows(const void* logits, int is_bf16, i64 stride_b, i64 stri
             }
             i64 off = (i64)b * stride_b + (i64)t * stride_t;
             const double* zr;
-            if (is_bf16) { widen_row((const uint16_t*)logits + off, V, z); zr = z; }
+            if (is_bf16) { widen_row((const uint16_t*)logits + off, V, z, is_bf16); zr = z; }
             else zr = (const double*)logits + off;
             double lse = row_lse(zr, V);
             i64 y = ids[(i64)b * ids_stride_b + t];
@@ -281,4 +321,86 @@ void oracle_dlogits_rows(const void* logits, int is_bf16, i64 stride_b, i64 stri
         }
         free(z);
     }
+}
+
+/* Entropy of the softmax of every valid row (R13):  H = -sum_v p_v log p_v  with  p_v = exp(z_v - lse),
+ * in nats; a deleted entry (z_v = -inf, p_v = 0) adds 0; 0 at padded positions.  `dtype` as `is_bf16` above. */
+void oracle_token_entropy(const void* logits, int dtype, i64 stride_b, i64 stride_t,
+                          const int32_t* lengths, int B, int T, i64 V, double* out_h)
+{
+    i64 rows = (i64)B * T;
+#pragma omp parallel
+    {
+        double* z = (double*)malloc(sizeof(double) * (size_t)V);
+#pragma omp for schedule(dynamic, 4)
+        for (i64 r = 0; r < rows; ++r) {
+            int b = (int)(r / T), t = (int)(r % T);
+            if (t >= lengths[b]) { out_h[r] = 0.0; continue; }
+            i64 off = (i64)b * stride_b + (i64)t * stride_t;
+            const double* zr;
+            if (dtype) { widen_row((const uint16_t*)logits + off, V, z, dtype); zr = z; }
+            else zr = (const double*)logits + off;
+            double lse = row_lse(zr, V);
+            double h = 0.0;
+            for (i64 v = 0; v < V; ++v) {
+                if (zr[v] == -INFINITY) continue;
+                double logp = zr[v] - lse;
+                h -= exp(logp) * logp;
+            }
+            out_h[r] = h;
+        }
+        free(z);
+    }
+}
+
+/* Monitors of the policy step over the valid tokens (R14, R15), from the new and old log-probs:
+ *   approx_kl = (1/N) sum (rho - 1 - log rho),   clip_frac = (1/N) #{ -A*clip(rho) > -A*rho },
+ * rho = exp(lp_new - lp_old).  Both 0 if N = 0. */
+void oracle_ppo_stats(const double* lp_new, const double* lp_old, const double* adv,
+                      const int32_t* lengths, int B, int T, double clip_eps,
+                      double* out_approx_kl, double* out_clip_frac)
+{
+    i64 N = 0, n_clipped = 0;
+    long double kl = 0.0L;
+    for (int b = 0; b < B; ++b) {
+        int len = lengths[b];
+        N += len;
+        for (int t = 0; t < len; ++t) {
+            i64 i = (i64)b * T + t;
+            double d = lp_new[i] - lp_old[i];
+            double rho = exp(d);
+            kl += (rho - 1.0) - d;
+            double unclipped = -adv[i] * rho;
+            double clipped = -adv[i] * clip_to(rho, 1.0 - clip_eps, 1.0 + clip_eps);
+            if (clipped > unclipped) ++n_clipped;
+        }
+    }
+    *out_approx_kl = N > 0 ? (double)(kl / (long double)N) : 0.0;
+    *out_clip_frac = N > 0 ? (double)n_clipped / (double)N : 0.0;
+}
+
+/* Advantage whitening over the valid tokens of the whole batch (R16): two passes, mean then
+ * population variance;  out = (A - mean) / sqrt(var + eps)  at valid positions, 0 elsewhere. */
+void oracle_whiten(const double* adv, const int32_t* lengths, int B, int T, double eps, double* out)
+{
+    i64 N = 0;
+    long double sum = 0.0L;
+    for (int b = 0; b < B; ++b) {
+        N += lengths[b];
+        for (int t = 0; t < lengths[b]; ++t) sum += adv[(i64)b * T + t];
+    }
+    double mean = N > 0 ? (double)(sum / (long double)N) : 0.0;
+    long double ss = 0.0L;
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < lengths[b]; ++t) {
+            double d = adv[(i64)b * T + t] - mean;
+            ss += d * d;
+        }
+    double var = N > 0 ? (double)(ss / (long double)N) : 0.0;
+    double denom = sqrt(var + eps);
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < T; ++t) {
+            i64 i = (i64)b * T + t;
+            out[i] = (t < lengths[b] && denom > 0.0) ? (adv[i] - mean) / denom : 0.0;
+        }
 }
