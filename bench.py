@@ -1,11 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the token-level PPO path: response tokens/s and achieved HBM bandwidth.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload opt] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|opt|...] [--impl ours|reference]
 
 One step is one pass of the whole path over one synthetic batch that is resident in HBM:
 log-probs of the actor logits and of the reference logits, the KL-penalised reward, GAE, and the
 fused PPO loss forward/backward that writes bf16 dlogits.  The line printed at the end is JSON.
+
+With --workload all (the default) the headline numbers (value, ms_per_step, e2e) are those of the
+OPT-shaped workload, exactly K steps timed; the Llama-2-shaped, large-vocabulary and ragged
+workloads are then timed the same way with step counts of their own, and every workload gets an
+entry in "roofline_by_workload".  Per workload there are two timed passes: the headline pass (K
+steps back to back, no events in between, so that each launch overlaps the tail of the one before
+it) and a detail pass in which every experience call and every loss call is bracketed by CUDA
+events on the launch stream, repeated until at least half a second has been timed.
 
 --impl reference times the float64 CPU oracle (plain C, OpenMP over rows) on the host cores on
 the same workload; it is a deliberately slow program, reported as a baseline, not a target.
@@ -28,11 +36,16 @@ if ROOT not in sys.path:
 METRIC = "fused logprob+PPO fwd/bwd: logit GB/s vs HBM peak; response tokens/s"
 UNIT = "response tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-EVENT_EVERY = 8            # steps between two event-timed loss launches inside the timed region
+NOMINAL_HBM_GBS = 8000.0       # the "roughly 8 TB/s" of the hardware's data sheet, for the second fraction
+DETAIL_MIN_MS = 500.0          # the detail pass repeats its K steps until this much has been timed
+DETAIL_MIN_LAUNCHES = 20
+ALL_WORKLOADS = ("opt", "llama2", "large_vocab", "ragged")
+# steps per timed pass of the workloads other than the headline one (about 0.5 s each)
+AUX_STEPS = {"llama2": 1000, "large_vocab": 100, "ragged": 120, "gpt2": 1500, "opt": 2000, "tiny": 2000}
 
-# DRAM bytes per launch of the loss kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
-# ncu capture summarised under profiles/, valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"sources_sha256": "32f96756e0de2479", "workload": "opt", "bytes_per_launch": 655180032}
+# DRAM bytes per launch of the loss kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# captures summarised under profiles/, valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {"sources_sha256": "", "bytes_per_launch": {}}
 
 
 def sources_digest() -> str:
@@ -53,7 +66,7 @@ def hbm_peak():
 
 class ClockSampler:
     """Samples SM clock, power and clock-event reasons of one GPU while a region runs (read-only queries):
-    through NVML in a thread of this process every 20 ms, or, where the NVML module is missing, through an
+    through NVML in a thread of this process every 10 ms, or, where the NVML module is missing, through an
     nvidia-smi child process every 100 ms."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -87,7 +100,7 @@ class ClockSampler:
                                       {n for n, m in self.MASKS.items() if mask & m}))
                 except Exception:
                     pass
-                if self._stop.wait(0.02):
+                if self._stop.wait(0.01):
                     return
 
         self.thread = threading.Thread(target=loop, daemon=True)
@@ -98,7 +111,7 @@ class ClockSampler:
             import pynvml as nvml
             nvml.nvmlInit()
             self._nvml_loop(nvml, nvml.nvmlDeviceGetHandleByIndex(self.index))
-            self.how = "nvml, 20 ms"
+            self.how = "nvml, 10 ms"
             return
         except Exception:
             self.thread = None
@@ -134,7 +147,12 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML module and no nvidia-smi"]}
         sm = sorted(r[0] for r in self.rows)
         reasons = set().union(*[r[3] for r in self.rows]) if self.rows else set()
+        bins = {}
+        for v in sm:                                       # samples binned by SM clock, 100 MHz wide
+            key = "%d-%d" % (int(v // 100) * 100, int(v // 100) * 100 + 99)
+            bins[key] = bins.get(key, 0) + 1
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max((r[1] for r in self.rows), default=None),
+                "sm_mhz_min": sm[0] if sm else None, "sm_mhz_bins": bins,
                 "power_w_max": max((r[2] for r in self.rows), default=None), "samples": len(sm),
                 "reasons": sorted(reasons), "sampled_by": self.how}
 
@@ -154,10 +172,10 @@ def visible_gpu_index(local_rank: int) -> int:
 class Path:
     """All buffers of one step, resident on the device, and the step itself (C-ABI calls only)."""
 
-    def __init__(self, w, batch, dev, fused=True, in_place=False):
+    def __init__(self, w, batch, dev, fused=True, in_place=False, global_mean=False):
         import torch
-        from paper_2410_15651_b200 import binding
-        self.b, self.w, self.binding = batch, w, binding
+        from paper_2410_15651_b200 import binding, parallel
+        self.b, self.w, self.binding, self.parallel = batch, w, binding, parallel
         B, T = w.B, w.T
         self.ws = binding.workspace(B, T, dev)
         f = lambda: torch.empty((B, T), dtype=torch.float32, device=dev)
@@ -166,6 +184,8 @@ class Path:
         self.exp.lp_actor, self.exp.lp_ref, self.exp.rewards = self.lp_act, self.lp_ref, self.rewards
         self.exp.adv, self.exp.returns = self.adv, self.ret
         self.fused = fused
+        self.global_mean = global_mean
+        self.batch_loss = None
         # in place: the gradient overwrites the logits it was computed from.  The loss call then gets a copy of
         # the actor logits of its own, so that the experience phase of the next step still reads logits; after
         # the first step that copy holds gradients, which costs the same traffic to read.
@@ -178,33 +198,188 @@ class Path:
         self.lp_old = (cur + batch["lp_old_noise"] * mask).contiguous()
         self.launches_per_step = 3 if fused else 5      # kernels of this library per step
 
-    def step(self, ev=None):
+    def experience(self):
         b, w, k = self.b, self.w, self.binding
         if self.fused:
-            # experience phase in one launch; the KL term uses the old-policy log-probs of the workload
+            # experience phase in one call; the KL term uses the old-policy log-probs of the workload
             k.experience(b["actor"], b["ref"], b["ids"], b["lengths"], b["score"], b["values_old"], w.beta_kl,
                          w.reward_clip, w.gamma, w.lam, self.ws, self.exp, lp_old=self.lp_old)
         else:
-            self._experience_separate()
+            k.gather_logprobs(b["actor"], b["ids"], b["lengths"], self.ws, self.lp_act)
+            k.gather_logprobs(b["ref"], b["ids"], b["lengths"], self.ws, self.lp_ref)
+            k.kl_reward(self.lp_old, self.lp_ref, b["score"], b["lengths"], w.beta_kl, w.reward_clip, self.rewards)
+            k.gae(self.rewards, b["values_old"], b["lengths"], w.gamma, w.lam, self.adv, self.ret)
+
+    def loss(self):
+        b, w, k = self.b, self.w, self.binding
+        grad_scale = float(self.N)                       # gradients of the token sum: O(1) entries
+        n_local = n_global = self.N
+        if self.global_mean:
+            # data parallel with one token mean over all ranks: all-reduce of the token counts before the loss call
+            n_local, n_global = self.parallel.token_counts(b["lengths"])
+            grad_scale = self.parallel.grad_scale_for_global_mean(n_local, n_global, upstream=float(n_global))
+        k.ppo_loss_fwd_bwd(self.loss_logits, b["ids"], b["lengths"], self.lp_old, self.adv, b["values_new"],
+                           b["values_old"], self.ret, w.clip_eps, w.value_clip, grad_scale, self.ws, self.out)
+        if self.global_mean:
+            self.batch_loss = self.parallel.combine_losses(self.out.loss, n_local, n_global)
+
+    def step(self, ev=None):
         if ev is not None:
             ev[0].record()
-        k.ppo_loss_fwd_bwd(self.loss_logits, b["ids"], b["lengths"], self.lp_old, self.adv, b["values_new"],
-                           b["values_old"], self.ret, w.clip_eps, w.value_clip, float(self.N), self.ws, self.out)
+        self.experience()
         if ev is not None:
             ev[1].record()
+        self.loss()
+        if ev is not None:
+            ev[2].record()
 
-    def _experience_separate(self):
-        b, w, k = self.b, self.w, self.binding
-        k.gather_logprobs(b["actor"], b["ids"], b["lengths"], self.ws, self.lp_act)
-        k.gather_logprobs(b["ref"], b["ids"], b["lengths"], self.ws, self.lp_ref)
-        k.kl_reward(self.lp_old, self.lp_ref, b["score"], b["lengths"], w.beta_kl, w.reward_clip, self.rewards)
-        k.gae(self.rewards, b["values_old"], b["lengths"], w.gamma, w.lam, self.adv, self.ret)
+
+def stats(xs):
+    xs = sorted(xs)
+    n = len(xs)
+    return {"median": xs[n // 2], "best": xs[0], "mean": sum(xs) / n, "n": n}
+
+
+def measure_workload(name, args, K, dev, rank, local_rank, world, with_e2e):
+    """Times one workload; returns the pieces of the JSON line that belong to it."""
+    import torch
+    import torch.distributed as dist
+    from paper_2410_15651_b200 import binding, inputs, parallel
+
+    w = inputs.scaled(inputs.WORKLOADS[name], seed=inputs.WORKLOADS[name].seed + 1000 * rank)
+    if args.sequences > 0:
+        w = inputs.scaled(w, B=args.sequences)
+    batch = inputs.make_batch(w, device=dev)
+    path = Path(w, batch, dev, fused=not args.separate_calls, in_place=args.in_place, global_mean=args.global_mean)
+    B, T, V = w.B, w.T, w.V
+    n_valid = path.N
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        path.step()
+    assert binding.poll_status(path.ws) == 0
+
+    # ---- headline pass: exactly K steps, one pair of CUDA events on the launching stream around all of them
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sync_all()
+    mem_before = (torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev))
+    sampler.start()
+    t0.record()
+    for i in range(K):
+        path.step()
+    t1.record()
+    sync_all()
+    mem_after = (torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev))
+    elapsed_ms = t0.elapsed_time(t1)
+    assert binding.poll_status(path.ws) == 0
+
+    # ---- detail pass: every experience call and every loss call between events; K steps, repeated until at
+    # least DETAIL_MIN_MS have been timed (an event between two launches keeps the second from starting its
+    # set-up under the tail of the first, so these steps are a little slower than the headline ones)
+    exp_ms, loss_ms, detail_total = [], [], 0.0
+    while detail_total < DETAIL_MIN_MS or len(loss_ms) < DETAIL_MIN_LAUNCHES:
+        evs = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(K)]
+        for i in range(K):
+            path.step(evs[i])
+        torch.cuda.synchronize(dev)
+        for a, b, c in evs:
+            exp_ms.append(a.elapsed_time(b))
+            loss_ms.append(b.elapsed_time(c))
+        detail_total += evs[0][0].elapsed_time(evs[-1][2])
+        if len(loss_ms) >= 20000:
+            break
+    sync_all()
+    clocks = sampler.stop()
+    assert binding.poll_status(path.ws) == 0
+    exp_s, loss_s = stats(exp_ms), stats(loss_ms)
+
+    # whole-job numbers: the slowest rank's time, the tokens of all ranks
+    elapsed_ms = parallel.max_over_ranks(elapsed_ms, dev)
+    loss_med = parallel.max_over_ranks(loss_s["median"], dev)
+    exp_med = parallel.max_over_ranks(exp_s["median"], dev)
+    total_tokens = parallel.sum_over_ranks(float(n_valid), dev)
+    ms_per_step = elapsed_ms / K
+    value = total_tokens / (ms_per_step * 1e-3)
+
+    peak, peak_src = hbm_peak()
+    loss_bytes = 2.0 * V * n_valid + 2.0 * V * B * T          # logits read on valid rows + dlogits written on all rows
+    exp_bytes = 2 * (2.0 * V * n_valid)                       # actor and reference logits read on valid rows
+    step_bytes = loss_bytes + exp_bytes
+    achieved = loss_bytes / (loss_med * 1e-3) / 1e9
+    exp_achieved = exp_bytes / (exp_med * 1e-3) / 1e9
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["sources_sha256"] == sources_digest():
+        traffic = NCU_TRAFFIC["bytes_per_launch"].get(name)
+
+    res = {
+        "name": name, "value": value, "ms_per_step": ms_per_step, "n_valid": n_valid, "clocks": clocks,
+        "launches": path.launches_per_step * K, "B": B, "T": T, "V": V,
+        "workspace_bytes": int(path.ws.numel()), "mem": (mem_before, mem_after), "step_bytes": step_bytes,
+        "roofline": {
+            "bound": "hbm", "kernel": "rlhf_ppo_loss_fwd_bwd (one launch: row kernel with fused finalisation)",
+            "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "frac_of_8000": achieved / NOMINAL_HBM_GBS, "peak_source": peak_src, "traffic": traffic,
+            "ms_per_launch": loss_med, "ms_per_launch_best": loss_s["best"], "ms_per_launch_mean": loss_s["mean"],
+            "launches_timed": loss_s["n"], "algorithmic_bytes_per_launch": loss_bytes,
+            "step_gbs": step_gbs, "step_frac": step_gbs / peak,
+            "note": ("frac is the loss call alone between two events; gradient lines that it leaves dirty in the "
+                     "L2 are written back during the next kernel, so traffic can be below the algorithmic bytes and "
+                     "step_frac (all three launches of a step, headline pass) is what a caller sees"),
+        },
+        "s1": {
+            "bound": "hbm", "kernel": "rlhf_experience (dual log-prob kernel + reward/GAE kernel)",
+            "achieved": exp_achieved, "peak": peak, "unit": "GB/s", "frac": exp_achieved / peak,
+            "frac_of_8000": exp_achieved / NOMINAL_HBM_GBS, "ms_per_call": exp_med,
+            "ms_per_call_best": exp_s["best"], "calls_timed": exp_s["n"], "algorithmic_bytes_per_call": exp_bytes,
+        },
+    }
+
+    if with_e2e:
+        # ---- end to end: inputs start in pinned host memory, losses are read back, every step
+        host = {k: batch[k].cpu().pin_memory() for k in ("actor", "ref", "ids", "lengths", "values_old",
+                                                          "values_new", "score")}
+        host["lp_old"] = path.lp_old.cpu().pin_memory()
+        loss_host = torch.empty(2, dtype=torch.float32).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = loss_host.numel() * 4
+        e_steps = max(3, min(20, K))
+
+        def e2e_step():
+            for k_ in ("actor", "ref", "ids", "lengths", "values_old", "values_new", "score"):
+                batch[k_].copy_(host[k_], non_blocking=True)
+            path.lp_old.copy_(host["lp_old"], non_blocking=True)
+            path.step()
+            loss_host.copy_(path.out.loss, non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e_steps):
+            e2e_step()
+        e1.record()
+        sync_all()
+        e2e_ms = parallel.max_over_ranks(e0.elapsed_time(e1), dev)
+        res["e2e"] = {"value": total_tokens / (e2e_ms / e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "steps": e_steps,
+                      "note": "bound by the host-to-device copy of the logits; a caller normally has them on the device"}
+    del path, batch
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2410_15651_b200 import binding, inputs, parallel
+    from paper_2410_15651_b200 import binding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -219,116 +394,54 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     binding.lib()                                              # fail here, loudly, if not built
-    w = inputs.scaled(inputs.WORKLOADS[args.workload], seed=inputs.WORKLOADS[args.workload].seed + 1000 * rank)
-    if args.sequences > 0:
-        w = inputs.scaled(w, B=args.sequences)
-    batch = inputs.make_batch(w, device=dev)
-    path = Path(w, batch, dev, fused=not args.separate_calls, in_place=args.in_place)
-    B, T, V = w.B, w.T, w.V
-    n_valid = path.N
+    names = list(ALL_WORKLOADS) if args.workload == "all" else [args.workload]
+    results = {}
+    for i, name in enumerate(names):
+        K = args.steps if i == 0 else (args.aux_steps or AUX_STEPS[name])
+        results[name] = measure_workload(name, args, K, dev, rank, local_rank, world, with_e2e=(i == 0))
+    head = results[names[0]]
 
-    def sync_all():
-        torch.cuda.synchronize(dev)
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize(dev)
+    # the top-level roofline: the workload whose loss launch is furthest below the peak (all have V >= 32000)
+    worst = min((r for r in results.values() if r["V"] >= 32000), key=lambda r: r["roofline"]["frac"], default=head)
+    roofline = dict(worst["roofline"])
+    roofline["workload"] = worst["name"]
+    by_workload = {}
+    for n, r in results.items():
+        by_workload[n] = {"shape": f"B={r['B']} T={r['T']} V={r['V']}", "response_tokens": r["n_valid"],
+                          "ms_per_step": r["ms_per_step"], "tokens_per_s": r["value"],
+                          "s4": {k: r["roofline"][k] for k in ("achieved", "frac", "frac_of_8000", "ms_per_launch",
+                                                               "ms_per_launch_best", "launches_timed", "traffic",
+                                                               "algorithmic_bytes_per_launch")},
+                          "s1": {k: r["s1"][k] for k in ("achieved", "frac", "frac_of_8000", "ms_per_call",
+                                                         "ms_per_call_best", "calls_timed")},
+                          "step_gbs": r["roofline"]["step_gbs"], "step_frac": r["roofline"]["step_frac"],
+                          "clocks": r["clocks"]}
 
-    for _ in range(args.warmup):
-        path.step()
-    assert binding.poll_status(path.ws) == 0
-
-    # ---- device-resident throughput: exactly K steps, CUDA events on the launching stream
-    K = args.steps
-    # The loss launch is bracketed by events on every EVENT_EVERY-th step only: an event between two launches
-    # keeps the second from starting its set-up under the tail of the first (programmatic dependent launch).
-    timed = [i for i in range(K) if i % EVENT_EVERY == 0]
-    inner = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for i in timed}
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    sync_all()
-    mem_before = (torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev))
-    sampler.start()
-    t0.record()
-    for i in range(K):
-        path.step(inner.get(i))
-    t1.record()
-    sync_all()
-    clocks = sampler.stop()
-    mem_after = (torch.cuda.memory_allocated(dev), torch.cuda.memory_reserved(dev))
-    elapsed_ms = t0.elapsed_time(t1)
-    loss_ms = sum(a.elapsed_time(b) for a, b in inner.values()) / len(inner)
-    assert binding.poll_status(path.ws) == 0
-
-    # whole-job numbers: the slowest rank's time, the tokens of all ranks
-    elapsed_ms = parallel.max_over_ranks(elapsed_ms, dev)
-    loss_ms = parallel.max_over_ranks(loss_ms, dev)
-    total_tokens = parallel.sum_over_ranks(float(n_valid), dev)
-    ms_per_step = elapsed_ms / K
-    value = total_tokens / (ms_per_step * 1e-3)
-
-    # ---- end to end: inputs start in pinned host memory, losses are read back, every step
-    host = {k: batch[k].cpu().pin_memory() for k in ("actor", "ref", "ids", "lengths", "values_old",
-                                                      "values_new", "score")}
-    host["lp_old"] = path.lp_old.cpu().pin_memory()
-    loss_host = torch.empty(2, dtype=torch.float32).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in host.values())
-    d2h = loss_host.numel() * 4
-    e_steps = max(3, min(20, K))
-
-    def e2e_step():
-        for k_ in ("actor", "ref", "ids", "lengths", "values_old", "values_new", "score"):
-            batch[k_].copy_(host[k_], non_blocking=True)
-        path.lp_old.copy_(host["lp_old"], non_blocking=True)
-        path.step()
-        loss_host.copy_(path.out.loss, non_blocking=True)
-
-    for _ in range(2):
-        e2e_step()
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e_steps):
-        e2e_step()
-    e1.record()
-    sync_all()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = parallel.max_over_ranks(e2e_ms, dev)
-    e2e_value = total_tokens / (e2e_ms / e_steps * 1e-3)
-
-    # ---- roofline of the dominant kernel (the loss forward/backward)
-    peak, peak_src = hbm_peak()
-    loss_bytes = 2.0 * V * n_valid + 2.0 * V * B * T          # logits read on valid rows + dlogits written on all rows
-    achieved = loss_bytes / (loss_ms * 1e-3) / 1e9
-    traffic = None
-    if NCU_TRAFFIC["sources_sha256"] == sources_digest() and NCU_TRAFFIC["workload"] == args.workload:
-        traffic = NCU_TRAFFIC["bytes_per_launch"]
-    step_bytes = loss_bytes + 2 * (2.0 * V * n_valid)         # + the two log-prob passes
-
+    B, T, V = head["B"], head["T"], head["V"]
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: B={B} T={T} V={V} bf16 logits, {n_valid} response tokens per GPU",
-                   "l2": "inputs larger than L2 (%.2f GB touched per step)" % (step_bytes / 1e9 + 0.0),
-                   "multi_gpu": "independent batch per rank, no data-path collective",
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{head['name']}: B={B} T={T} V={V} bf16 logits, {head['n_valid']} response tokens per GPU",
+                   "also_timed": [n for n in names[1:]],
+                   "l2": "inputs larger than L2 (%.2f GB touched per step)" % (head["step_bytes"] / 1e9),
+                   "multi_gpu": ("one batch shard per rank; token counts all-reduced (NCCL) before the loss call, "
+                                 "losses combined by a token-weighted all-reduce after it" if args.global_mean else
+                                 "independent batch per rank, no data-path collective"),
                    "dlogits": "in place (over a copy of the logits)" if args.in_place else "separate bf16 [B,T,V] buffer",
-                   "workspace_bytes": int(path.ws.numel()), "workspace_bound_16BT_plus_64K": 16 * B * T + 65536,
-                   "torch_allocated_bytes_before_after": [mem_before[0], mem_after[0]],
-                   "torch_reserved_bytes_before_after": [mem_before[1], mem_after[1]],
+                   "workspace_bytes": head["workspace_bytes"], "workspace_bound_16BT_plus_64K": 16 * B * T + 65536,
+                   "torch_allocated_bytes_before_after": [head["mem"][0][0], head["mem"][1][0]],
+                   "torch_reserved_bytes_before_after": [head["mem"][0][1], head["mem"][1][1]],
                    "calls_per_step": ("rlhf_gather_logprobs x2, rlhf_kl_reward, rlhf_gae, rlhf_ppo_loss_fwd_bwd"
                                       if args.separate_calls else "rlhf_experience, rlhf_ppo_loss_fwd_bwd")},
-        "clocks": clocks, "gpu_launches": path.launches_per_step * K,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e_steps},
-        "roofline": {"bound": "hbm", "kernel": "rlhf_ppo_loss_fwd_bwd (one launch: row kernel with fused finalisation)",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": peak_src, "traffic": traffic, "ms_per_launch": loss_ms,
-                     "launches_timed": len(inner),
-                     "algorithmic_bytes_per_launch": loss_bytes,
-                     "step_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9},
+        "clocks": head["clocks"], "gpu_launches": head["launches"],
+        "e2e": head["e2e"],
+        "roofline": roofline,
+        "roofline_s1": head["s1"],
+        "roofline_by_workload": by_workload,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=15.0)
+        line["cpu_baseline"] = cpu_baseline(names[0], budget_s=12.0)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -371,23 +484,33 @@ def oracle_inputs(workload: str, n_seq: int):
 
 
 def cpu_baseline(workload: str, budget_s: float):
-    """The oracle, as it stands, on a bounded sample of the workload: whole sequences, as many as fit
-    in about `budget_s` seconds of wall time on the host cores."""
+    """The oracle, as it stands, on a bounded sample of the workload: whole sequences, as many as fit in about
+    `budget_s` seconds of wall time with all host threads, then about a third of that again with one thread."""
     import oracle
     oracle.build()
     w, bn = oracle_inputs(workload, n_seq=2)
-    t0 = time.perf_counter()
-    n = oracle_pass(oracle, w, bn, [0])
-    dt = time.perf_counter() - t0
-    reps = max(1, int(budget_s / max(dt, 1e-3)))
-    t0 = time.perf_counter()
-    tokens = 0
-    for i in range(reps):
-        tokens += oracle_pass(oracle, w, bn, [i % w.B])
-    dt = time.perf_counter() - t0
-    return {"value": tokens / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    all_threads = oracle.num_threads()
+
+    def timed(budget):
+        t0 = time.perf_counter()
+        oracle_pass(oracle, w, bn, [0])
+        dt = time.perf_counter() - t0
+        reps = max(1, int(budget / max(dt, 1e-3)))
+        t0 = time.perf_counter()
+        tokens = 0
+        for i in range(reps):
+            tokens += oracle_pass(oracle, w, bn, [i % w.B])
+        return tokens, reps, time.perf_counter() - t0
+
+    tokens, reps, dt = timed(budget_s)
+    oracle.set_num_threads(1)
+    tokens1, reps1, dt1 = timed(budget_s / 3)
+    oracle.set_num_threads(all_threads)
+    return {"value": tokens / dt, "unit": UNIT, "cores": all_threads, "nproc": os.cpu_count(), "kind": "oracle",
             "sample": f"{reps} sequence passes of the {workload} workload (T={w.T}, V={w.V}), "
-                      f"{tokens} response tokens, {dt:.1f} s"}
+                      f"{tokens} response tokens, {dt:.1f} s",
+            "one_thread": {"value": tokens1 / dt1, "cores": 1,
+                           "sample": f"{reps1} sequence passes, {tokens1} response tokens, {dt1:.1f} s"}}
 
 
 def run_reference(args):
@@ -397,8 +520,9 @@ def run_reference(args):
     import oracle
     oracle.build()
     from paper_2410_15651_b200 import inputs
-    w, bn = oracle_inputs(args.workload, n_seq=2)
-    full = inputs.WORKLOADS[args.workload]
+    name = "opt" if args.workload == "all" else args.workload
+    w, bn = oracle_inputs(name, n_seq=2)
+    full = inputs.WORKLOADS[name]
     for i in range(min(args.warmup, 2)):
         oracle_pass(oracle, w, bn, [0])
     t0 = time.perf_counter()
@@ -408,15 +532,15 @@ def run_reference(args):
         tokens += oracle_pass(oracle, w, bn, [i % w.B])
     dt = time.perf_counter() - t0
     value = tokens / dt
-    sample = (f"each step = one sequence of the {args.workload} workload (T={w.T}, V={w.V}); "
+    sample = (f"each step = one sequence of the {name} workload (T={w.T}, V={w.V}); "
               f"{steps} steps timed, {tokens} response tokens")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": dt / steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: B={full.B} T={full.T} V={full.V} bf16 logits (sampled by sequence)"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                         "sample": sample},
+        "config": {"workload": f"{name}: B={full.B} T={full.T} V={full.V} bf16 logits (sampled by sequence)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "nproc": os.cpu_count(),
+                         "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -424,16 +548,21 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="opt", choices=["tiny", "opt", "llama2", "large_vocab", "ragged", "gpt2"])
+    ap.add_argument("--workload", default="all",
+                    choices=["all", "tiny", "opt", "llama2", "large_vocab", "ragged", "gpt2"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sequences", type=int, default=0,
                     help="override the number of sequences B of the workload (smaller cases for profiling)")
+    ap.add_argument("--aux-steps", type=int, default=0,
+                    help="steps per timed pass of the workloads after the first (default: about 0.5 s each)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--in-place", action="store_true", help="dlogits overwrite the logits given to the loss call")
     ap.add_argument("--separate-calls", action="store_true",
                     help="experience phase as four calls (2 x gather_logprobs, kl_reward, gae) instead of rlhf_experience")
+    ap.add_argument("--global-mean", action="store_true",
+                    help="with --gpus N: one token mean over all ranks (token counts and losses all-reduced every step)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

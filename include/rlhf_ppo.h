@@ -13,6 +13,7 @@
  *   rlhf_gae                advantages and returns from rewards and critic values
  *   rlhf_ppo_loss_fwd_bwd   clipped policy and value loss, gradient w.r.t. the logits and values
  *   rlhf_experience         the first three together (both log-prob passes in one kernel, reward + GAE in another)
+ *   rlhf_whiten_advantages  optional masked whitening of the advantages between steps 3 and 4
  *
  * The paper gives these quantities in prose only; the formulas are the standard definitions and
  * are written out beside each function.
@@ -38,8 +39,11 @@
  *  - Return value: an rlhf_status_t.  Errors the host can see (null pointers, sizes, strides,
  *    scalars out of range, workspace too small) are returned at once and nothing is launched.
  *    Errors only the device can see (an id outside [0,V), a length outside [0,T], a bounded wait
- *    that ran out) never fault: the offending token is treated as padding (length clamped), the
- *    code is OR-ed into the first word of the workspace, and rlhf_poll_status reports it.
+ *    that ran out) never fault; the code is OR-ed into the first word of the workspace, and
+ *    rlhf_poll_status reports it.  A length outside [0,T] is clamped to that range.  A token
+ *    whose id is outside [0,V) gets log-prob 0, policy-loss term 0 and an all-zero dlogits row;
+ *    it still counts in N, and its value-loss term and dvalues entry (which do not depend on the
+ *    id) are computed as for any valid token.
  *  - Arithmetic: fp32 throughout (exp/log of the softmax in base 2 with the hardware ex2); bf16
  *    outputs are rounded to nearest even.  Results do not depend on the order in which rows are
  *    scheduled: the loss is reduced in a fixed order, without floating-point atomics.
@@ -56,7 +60,7 @@ extern "C" {
 typedef enum {
     RLHF_OK = 0,
     RLHF_ERR_NULL = 1,          /* a required pointer is NULL */
-    RLHF_ERR_SHAPE = 2,         /* B, T or V <= 0, or B*T too large */
+    RLHF_ERR_SHAPE = 2,         /* B, T or V <= 0, or B*T above 2^29 */
     RLHF_ERR_ALIGN = 3,         /* a [B,T] array or the workspace is not aligned to its element / 256 B */
     RLHF_ERR_STRIDE = 4,        /* stride_t < V, negative stride, rows of different sequences overlap */
     RLHF_ERR_WORKSPACE = 5,     /* workspace smaller than rlhf_workspace_bytes(B,T) */
@@ -142,6 +146,19 @@ int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score,
  */
 int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, int B, int T,
              float gamma, float lambda, float* out_adv, float* out_returns, void* stream);
+
+/*
+ * Optional, between steps 3 and 4 -- advantage whitening over the whole batch (Section 2.1 leaves the
+ * normalisation of the advantages open; off unless the caller makes this call).  With N valid tokens,
+ *     mean = (1/N) sum A,   var = (1/N) sum (A - mean)^2,   out_adv = (A - mean) / sqrt(var + eps)
+ * at valid positions and 0 at padded ones; all zeros if N = 0 or var + eps = 0.  The sums are formed in
+ * double precision in a fixed order (no floating-point atomics), so the result is bit-stable.
+ *   adv       fp32 [B,T]; lengths int32 [B]                              read
+ *   out_adv   fp32 [B,T]                                                 written; may be adv itself
+ *   eps >= 0, finite.   workspace as for step 1.
+ */
+int rlhf_whiten_advantages(const float* adv, const int* lengths, int B, int T, float eps, float* out_adv,
+                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Steps 1-3 together -- the whole experience phase (Section 2.1: the inferences of the actor,

@@ -32,6 +32,7 @@ SIGNATURES = {
     "rlhf_gather_logprobs": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
     "rlhf_kl_reward": (_int, [_vp, _vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
     "rlhf_gae": (_int, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp, _vp]),
+    "rlhf_whiten_advantages": (_int, [_vp, _vp, _int, _int, _f32, _vp, _vp, _sz, _vp]),
     "rlhf_experience": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp,
                                _int, _int, _int, _f32, _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "rlhf_ppo_loss_fwd_bwd": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -192,6 +193,19 @@ def gae(rewards: torch.Tensor, values_old: torch.Tensor, lengths: torch.Tensor, 
     _check(lib().rlhf_gae(rewards.data_ptr(), values_old.data_ptr(), lengths.data_ptr(), B, T, gamma, lam,
                           out_adv.data_ptr(), out_returns.data_ptr(), _stream(rewards)), "rlhf_gae")
     return out_adv, out_returns
+
+
+def whiten_advantages(adv: torch.Tensor, lengths: torch.Tensor, eps: float, ws: torch.Tensor,
+                      out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    B, T = adv.shape
+    _bt(adv, B, T, "adv")
+    _lengths(lengths, B)
+    if out is None:
+        out = torch.empty_like(adv)
+    _bt(out, B, T, "out")
+    _check(lib().rlhf_whiten_advantages(adv.data_ptr(), lengths.data_ptr(), B, T, eps, out.data_ptr(),
+                                        ws.data_ptr(), ws.numel(), _stream(adv)), "rlhf_whiten_advantages")
+    return out
 
 
 class Experience:

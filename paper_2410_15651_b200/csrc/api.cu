@@ -13,6 +13,7 @@
 #include "kernels_generic.cuh"
 #include "kernels_ring.cuh"
 #include "kernels_dbuf.cuh"
+#include "kernels_creg.cuh"
 #include "kernels_warp.cuh"
 #include "kernels_small.cuh"
 
@@ -34,19 +35,24 @@ int cuda_fail(cudaError_t e, const char* what)
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
-// Workspace layout (bytes): [0,4) status flags, [4,8) finalisation ticket, [256, kRowLossOffset) block
+// Workspace layout (bytes): [0,4) status flags, [4,8) reduction ticket, [8,16) mean and 1/std of the
+// advantage whitening, [16,20) row counter of the loss kernel that deals its rows dynamically, [256, kRowLossOffset) block
 // partial sums of the two losses (2 doubles per block of the kernel that reduces them),
 // [kRowLossOffset, +4*B*T) per-token policy loss terms (kernels without the fused finalisation).
 constexpr size_t kPartialsOffset = 256;
 constexpr size_t kRowLossOffset = 24576;
 constexpr int kMaxFusedBlocks = (int)((kRowLossOffset - kPartialsOffset) / 16);   // block partials that fit the header
 
+constexpr long long kMaxTokens = 1ll << 29;
+
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 int check_shape(int B, int T, int V)
 {
     if (B <= 0 || T <= 0 || V <= 0) return RLHF_ERR_SHAPE;
-    if ((long long)B * (long long)T > (1ll << 30)) return RLHF_ERR_SHAPE;
+    // the log-prob kernel walks up to 2*B*T rows (two tensors in one launch) plus one grid stride with 32-bit
+    // indices, so B*T stays at or below 2^29
+    if ((long long)B * (long long)T > kMaxTokens) return RLHF_ERR_SHAPE;
     return RLHF_OK;
 }
 
@@ -87,20 +93,42 @@ bool rows_16B(const void* base, long long stride_b, long long stride_t, int V)
 
 // Launches `kernel` with programmatic stream serialisation allowed (see pdl_wait_prior_grid): the launch
 // itself and the kernel's set-up overlap the tail of the kernel before it in the stream.
-template <typename... Params, typename... Args>
-cudaError_t launch_kernel(void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, Args&&... args)
+// `cluster` > 1 launches the grid as thread-block clusters of that many blocks.
+void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute (&attr)[2], int grid, int block, size_t smem,
+                        int cluster, cudaStream_t s)
 {
-    cudaLaunchConfig_t cfg = {};
+    cfg = cudaLaunchConfig_t{};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (cluster > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+}
+
+template <typename... Params, typename... Args>
+cudaError_t launch_kernel_cluster(void (*kernel)(Params...), int grid, int block, size_t smem, int cluster,
+                                  cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    fill_launch_config(cfg, attr, grid, block, smem, cluster, s);
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
+template <typename... Params, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    return launch_kernel_cluster(kernel, grid, block, smem, 1, s, static_cast<Args&&>(args)...);
 }
 
 template <int NW, int U>
@@ -151,10 +179,108 @@ int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     return RLHF_OK;
 }
 
-// The loss row kernel for 16-byte aligned rows: two resident rows where that fits, else the chunk ring.
+// Loss kernel that keeps a row's exponentials on chip (kernels_creg.cuh): in registers if a consumer thread has at
+// most kRegVecsOnly vectors of a row, else in registers for its first kRegVecsTmem vectors and in tensor memory for
+// up to kTmemVecs more.  A block holds two buffers of its share of
+// a row; rows that do not fit twice are shared by a cluster of up to 4 blocks.
+constexpr int kCregWarps = 16;
+
+struct CregPlan {
+    int cluster = 0;            // blocks per cluster, 1..4; 0 = the kernel does not apply
+    unsigned slice_vecs = 0;
+    unsigned tmem_cols = 0;
+    int n_buf = 0;              // slice buffers per block
+    size_t smem_bytes = 0;
+};
+
+CregPlan plan_creg(unsigned row_bytes, const DeviceInfo& dev)
+{
+    CregPlan pl;
+    if (row_bytes < 16384 || row_bytes % 16 != 0) return pl;
+    const unsigned row_vecs = row_bytes / 16;
+    const unsigned cap = (unsigned)kCregWarps * 32 * (kRegVecsTmem + kTmemVecs);
+    for (int c = 1; c <= 4; ++c) {
+        const unsigned sv = (row_vecs + c - 1) / c;
+        if (sv > cap) continue;
+        int nb = kCregMaxBufs;
+        while (nb >= 2 && creg_smem_bytes(sv, kCregWarps, nb) + 2048 > (size_t)dev.max_smem_optin) --nb;
+        if (nb < 2) continue;
+        pl.cluster = c;
+        pl.slice_vecs = sv;
+        pl.tmem_cols = creg_tmem_cols(sv, kCregWarps);
+        pl.n_buf = nb;
+        pl.smem_bytes = creg_smem_bytes(sv, kCregWarps, nb);
+        return pl;
+    }
+    return pl;
+}
+
+// Clusters of the kernel that the device holds at once (one block per SM); looked up once per device and
+// cluster size.  It only sizes the persistent grid: a larger grid would still be correct.
+template <int NW, int C, bool kTmem>
+int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
+{
+    if (C == 1) { out = dev.sm_count; return RLHF_OK; }
+    static std::mutex mu;
+    static int cached[64] = {};
+    int d = 0;
+    RLHF_CUDA(cudaGetDevice(&d));
+    std::lock_guard<std::mutex> lock(mu);
+    if (d < 0 || d >= 64 || cached[d] == 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[2];
+        fill_launch_config(cfg, attr, dev.sm_count / C * C, NW * 32 + 32, pl.smem_bytes, C, nullptr);
+        RLHF_CUDA(cudaOccupancyMaxActiveClusters(&n, loss_creg_kernel<NW, C, kTmem>, &cfg));
+        if (n < 1) n = 1;
+        if (d < 0 || d >= 64) { out = n; return RLHF_OK; }
+        cached[d] = n;
+    }
+    out = cached[d];
+    return RLHF_OK;
+}
+
+template <int NW, int C, bool kTmem>
+int launch_creg(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cudaStream_t s)
+{
+    CregArgs ca{};
+    ca.row = a;
+    ca.row_bytes = 2u * (unsigned)a.V;
+    ca.slice_vecs = pl.slice_vecs;
+    ca.buf_stride = (unsigned)creg_buf_stride(pl.slice_vecs, NW);
+    ca.tmem_cols = pl.tmem_cols;
+    ca.n_buf = pl.n_buf;
+    ca.row_counter = (unsigned*)((char*)a.status + 16);
+    RLHF_CUDA(cudaFuncSetAttribute(loss_creg_kernel<NW, C, kTmem>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)pl.smem_bytes));
+    int clusters = 0;
+    if (int e = creg_resident_clusters<NW, C, kTmem>(pl, dev, clusters)) return e;
+    const long long rows = (long long)a.B * a.T;
+    const int grid = (int)std::min<long long>(rows, clusters) * C;
+    RLHF_CUDA(launch_kernel_cluster(loss_creg_kernel<NW, C, kTmem>, grid, NW * 32 + 32, pl.smem_bytes, C, s, ca));
+    return RLHF_OK;
+}
+
+template <int NW, bool kTmem>
+int launch_creg_cluster(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cudaStream_t s)
+{
+    switch (pl.cluster) {
+        case 1: return launch_creg<NW, 1, kTmem>(a, pl, dev, s);
+        case 2: return launch_creg<NW, 2, kTmem>(a, pl, dev, s);
+        case 3: return launch_creg<NW, 3, kTmem>(a, pl, dev, s);
+        default: return launch_creg<NW, 4, kTmem>(a, pl, dev, s);
+    }
+}
+
+// The loss row kernel for 16-byte aligned rows: exponentials in registers where the row (or its share in a
+// cluster) fits, else two resident rows, else the chunk ring.
 int launch_loss_rows(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 {
     const unsigned row_bytes = 2u * (unsigned)a.V;
+    const CregPlan cp = plan_creg(row_bytes, dev);
+    if (cp.cluster > 0)
+        return cp.tmem_cols != 0 ? launch_creg_cluster<kCregWarps, true>(a, cp, dev, s)
+                                 : launch_creg_cluster<kCregWarps, false>(a, cp, dev, s);
     if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false>(a, dev, s);
     const RingPlan pl = plan_ring(row_bytes, dev.smem_per_sm, dev.max_smem_optin);
     RingArgs ra{};
@@ -177,6 +303,34 @@ template <typename K>
 int keep_max_carveout(K kernel)
 {
     RLHF_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    return RLHF_OK;
+}
+
+// Host-side checks of the loss call's arguments, the workspace apart (shared by the two loss entry points).
+int check_loss_args(const void* logits, long long stride_b, long long stride_t, const long long* ids,
+                    long long ids_stride_b, const int* lengths, const float* lp_old, const float* adv,
+                    const float* values_new, const float* values_old, const float* returns, int B, int T, int V,
+                    float clip_eps, float value_clip, float grad_scale, const float* out_loss_pg,
+                    const float* out_loss_vf, const void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                    const float* out_dvalues, const float* out_lp_new)
+{
+    if (!logits || !ids || !lengths || !lp_old || !adv || !values_new || !values_old || !returns ||
+        !out_loss_pg || !out_loss_vf || !out_dlogits || !out_dvalues)
+        return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, V)) return e;
+    if (stride_b < 0 || stride_t < 0 || ids_stride_b < 0 || dl_stride_b < 0 || dl_stride_t < 0)
+        return RLHF_ERR_STRIDE;
+    if (T > 1 && (stride_t < V || dl_stride_t < V)) return RLHF_ERR_STRIDE;
+    if (B > 1 && dl_stride_b < (long long)(T - 1) * dl_stride_t + V) return RLHF_ERR_STRIDE;
+    if (out_dlogits == logits && (dl_stride_b != stride_b || dl_stride_t != stride_t)) return RLHF_ERR_STRIDE;
+    if (!(clip_eps > 0.f && clip_eps < 1.f) || !std::isfinite(value_clip) || value_clip < 0.f ||
+        !std::isfinite(grad_scale))
+        return RLHF_ERR_SCALAR;
+    if (!aligned(logits, 2) || !aligned(out_dlogits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) ||
+        !aligned(lp_old, 4) || !aligned(adv, 4) || !aligned(values_new, 4) || !aligned(values_old, 4) ||
+        !aligned(returns, 4) || !aligned(out_loss_pg, 4) || !aligned(out_loss_vf, 4) ||
+        !aligned(out_dvalues, 4) || (out_lp_new && !aligned(out_lp_new, 4)))
+        return RLHF_ERR_ALIGN;
     return RLHF_OK;
 }
 
@@ -287,6 +441,7 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
     a.lengths = lengths;
     a.B = B; a.T = T; a.V = V;
     a.status = (unsigned*)workspace;
+    a.wait_limit_ns = kWaitLimitNs;
     a.out_lp = out_logprobs;
 
     WarpArgs wa{};
@@ -337,6 +492,36 @@ int rlhf_gae(const float* rewards, const float* values_old, const int* lengths, 
     return launch_check("gae_kernel");
 }
 
+int rlhf_whiten_advantages(const float* adv, const int* lengths, int B, int T, float eps, float* out_adv,
+                           void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!adv || !lengths || !out_adv) return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, 1)) return e;
+    if (!std::isfinite(eps) || eps < 0.f) return RLHF_ERR_SCALAR;
+    if (!aligned(adv, 4) || !aligned(lengths, 4) || !aligned(out_adv, 4)) return RLHF_ERR_ALIGN;
+    if (int e = check_workspace(workspace, workspace_bytes, rlhf_workspace_bytes(B, T))) return e;
+    char* ws = (char*)workspace;
+    WhitenArgs w{};
+    w.adv = adv;
+    w.lengths = lengths;
+    w.B = B; w.T = T;
+    w.eps = eps;
+    w.out = out_adv;
+    w.ticket = (unsigned*)(ws + 4);
+    w.partials = (double*)(ws + kPartialsOffset);
+    w.mean_rstd = (float*)(ws + 8);
+    const long long total = (long long)B * T;
+    const int grid = (int)std::min<long long>((total + 4095) / 4096, kWhitenMaxBlocks);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (int e = keep_max_carveout(whiten_stats_kernel)) return e;
+    RLHF_CUDA(launch_kernel(whiten_stats_kernel, grid, kWhitenThreads, 0, s, w));
+    if (int e = launch_check("whiten_stats_kernel")) return e;
+    if (int e = keep_max_carveout(whiten_apply_kernel)) return e;
+    const int agrid = (int)std::min<long long>((total + 255) / 256, 1184);
+    RLHF_CUDA(launch_kernel(whiten_apply_kernel, agrid, 256, 0, s, w));
+    return launch_check("whiten_apply_kernel");
+}
+
 int rlhf_experience(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
                     const void* ref_logits, long long ref_stride_b, long long ref_stride_t,
                     const long long* ids, long long ids_stride_b, const int* lengths,
@@ -383,6 +568,7 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     wa.row.lengths = lengths;
     wa.row.B = B; wa.row.T = T; wa.row.V = V;
     wa.row.status = (unsigned*)workspace;
+    wa.row.wait_limit_ns = kWaitLimitNs;
     wa.row.out_lp = out_lp_actor;
     wa.logits2 = (const uint16_t*)ref_logits;
     wa.stride2_b = ref_stride_b;
@@ -413,23 +599,10 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
                           float* out_dvalues, float* out_lp_new,
                           void* workspace, size_t workspace_bytes, void* stream)
 {
-    if (!logits || !ids || !lengths || !lp_old || !adv || !values_new || !values_old || !returns ||
-        !out_loss_pg || !out_loss_vf || !out_dlogits || !out_dvalues)
-        return RLHF_ERR_NULL;
-    if (int e = check_shape(B, T, V)) return e;
-    if (stride_b < 0 || stride_t < 0 || ids_stride_b < 0 || dl_stride_b < 0 || dl_stride_t < 0)
-        return RLHF_ERR_STRIDE;
-    if (T > 1 && (stride_t < V || dl_stride_t < V)) return RLHF_ERR_STRIDE;
-    if (B > 1 && dl_stride_b < (long long)(T - 1) * dl_stride_t + V) return RLHF_ERR_STRIDE;
-    if (out_dlogits == logits && (dl_stride_b != stride_b || dl_stride_t != stride_t)) return RLHF_ERR_STRIDE;
-    if (!(clip_eps > 0.f && clip_eps < 1.f) || !std::isfinite(value_clip) || value_clip < 0.f ||
-        !std::isfinite(grad_scale))
-        return RLHF_ERR_SCALAR;
-    if (!aligned(logits, 2) || !aligned(out_dlogits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) ||
-        !aligned(lp_old, 4) || !aligned(adv, 4) || !aligned(values_new, 4) || !aligned(values_old, 4) ||
-        !aligned(returns, 4) || !aligned(out_loss_pg, 4) || !aligned(out_loss_vf, 4) ||
-        !aligned(out_dvalues, 4) || (out_lp_new && !aligned(out_lp_new, 4)))
-        return RLHF_ERR_ALIGN;
+    if (int e = check_loss_args(logits, stride_b, stride_t, ids, ids_stride_b, lengths, lp_old, adv, values_new,
+                                values_old, returns, B, T, V, clip_eps, value_clip, grad_scale, out_loss_pg,
+                                out_loss_vf, out_dlogits, dl_stride_b, dl_stride_t, out_dvalues, out_lp_new))
+        return e;
     if (int e = check_workspace(workspace, workspace_bytes, loss_workspace_bytes(B, T))) return e;
     DeviceInfo dev;
     if (int e = device_info(dev)) return e;
@@ -444,6 +617,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
     a.lengths = lengths;
     a.B = B; a.T = T; a.V = V;
     a.status = (unsigned*)ws;
+    a.wait_limit_ns = kWaitLimitNs;
     a.lp_old = lp_old;
     a.adv = adv;
     a.clip_eps = clip_eps;
@@ -558,11 +732,16 @@ extern "C" int rlhf_ppo_loss_fwd_bwd_noalloc(const void* logits, long long strid
     if (B <= 0 || T <= 0) return RLHF_ERR_SHAPE;
     if ((long long)B * (long long)T > (long long)RLHF_NOALLOC_MAX_TOKENS) return RLHF_ERR_TOO_LARGE;
     if (out_device_status && !aligned(out_device_status, 4)) return RLHF_ERR_ALIGN;
+    // every host-side check first: a refused call must not have queued anything on the stream
+    if (int e = check_loss_args(logits, stride_b, stride_t, ids, ids_stride_b, lengths, lp_old, adv, values_new,
+                                values_old, returns, B, T, V, clip_eps, value_clip, grad_scale, out_loss_pg,
+                                out_loss_vf, out_dlogits, dl_stride_b, dl_stride_t, out_dvalues, out_lp_new))
+        return e;
     void* scratch = nullptr;
     if (int e = noalloc_scratch(&scratch)) return e;
     cudaStream_t s = (cudaStream_t)stream;
-    // the status word and the reduction ticket must start at zero; the rest is written before it is read
-    RLHF_CUDA(cudaMemsetAsync(scratch, 0, 8, s));
+    // the status word, the reduction ticket and the row counter must start at zero; the rest is written before it is read
+    RLHF_CUDA(cudaMemsetAsync(scratch, 0, 32, s));
     int e = rlhf_ppo_loss_fwd_bwd(logits, stride_b, stride_t, ids, ids_stride_b, lengths, lp_old, adv,
                                   values_new, values_old, returns, B, T, V, clip_eps, value_clip, grad_scale,
                                   out_loss_pg, out_loss_vf, out_dlogits, dl_stride_b, dl_stride_t,

@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         unsigned char *drow0 = nullptr, *drow1 = nullptr;       // global rows the two buffers drain to
         auto drain = [&](long long i) {
             const int buf = (int)(i & 1);
-            mbar_wait(computed(buf), (uint32_t)(i >> 1) & 1u, p.status, aborted);
+            mbar_wait(computed(buf), (uint32_t)(i >> 1) & 1u, p.status, aborted, p.wait_limit_ns);
             if (aborted) return;
             const uint32_t srcb = buf_addr + (uint32_t)buf * da.row_stride;
             unsigned char* drow = buf ? drow1 : drow0;               // the row's first entry in global memory
@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
     for (long long k = blockIdx.x; k < N; k += G, ++i) {
         const int buf = (int)(i & 1), par = buf;
         const uint32_t use = (uint32_t)(i >> 1) & 1u;
-        mbar_wait(landed(buf, 0), use, p.status, aborted);
+        mbar_wait(landed(buf, 0), use, p.status, aborted, p.wait_limit_ns);
         RowInfo ri = s_row[buf];
         if (aborted) { ri.y = 0; ri.bad_id = 1; ri.flat = 0; }      // stale row info: touch nothing
         // where the row sits in the buffer: eoff entries of vector 0 precede it (kAny), vectors [0, row_vecs)
@@ -316,7 +316,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
             for (; j < j1; ++j) add_special(a, src[(size_t)j * kCons], j, zy);
         };
         sum_range(0, head_cnt);
-        mbar_wait(landed(buf, 1), use, p.status, aborted);
+        mbar_wait(landed(buf, 1), use, p.status, aborted, p.wait_limit_ns);
         sum_range(head_cnt, cnt);
         if (redo) {
             a = acc_empty();

@@ -16,6 +16,7 @@ struct RowArgs {
     const int* lengths;
     int B, T, V;
     unsigned* status;           // workspace word 0
+    unsigned long long wait_limit_ns;   // bound of every wait on a shared-memory barrier (row kernels with a producer)
     // step 1
     float* out_lp;
     // step 4

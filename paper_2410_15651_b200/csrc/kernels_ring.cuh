@@ -26,7 +26,7 @@
 namespace rlhf {
 
 constexpr int kZeroBytes = 4096;                       // zeroed buffer that feeds the bulk zero-fill
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default bound of a barrier wait: 2 s
 
 struct RingArgs {
     RowArgs row;
@@ -68,23 +68,24 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 // Bounded wait.  Returns false (after flagging the status word) if the phase did not complete in time.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, unsigned* status)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, unsigned* status, unsigned long long limit_ns)
 {
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
         for (int i = 0; i < 128; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (global_timer_ns() - t0 > limit_ns) {
             atomicOr(status, kErrTimeout);
             return false;
         }
     }
 }
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, unsigned* status, bool& aborted)
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, unsigned* status, bool& aborted,
+                                          unsigned long long limit_ns)
 {
     if (aborted) return;
     if (mbar_try_wait(bar, parity)) return;
-    if (!mbar_wait_slow(bar, parity, status)) aborted = true;
+    if (!mbar_wait_slow(bar, parity, status, limit_ns)) aborted = true;
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
@@ -385,7 +386,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
             const unsigned char* row = (const unsigned char*)(p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t);
             for (int j = 0; j < loads_per_row; ++j) {
                 const int c = j >= chunks ? j - chunks : j;
-                mbar_wait(empty_addr + 8u * slot, phase ^ 1u, p.status, aborted);
+                mbar_wait(empty_addr + 8u * slot, phase ^ 1u, p.status, aborted, p.wait_limit_ns);
                 if (aborted) break;
                 const uint32_t off = (uint32_t)c * kChunk;
                 const uint32_t bytes = min(kChunk, ra.row_bytes - off);
@@ -451,7 +452,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
         float Mref = kFloorM;
         const bool owner = (yvec % kCons) == (uint32_t)tid;      // this thread sums the generated token's vector
         for (int c = 0; c < chunks; ++c) {
-            mbar_wait(full_addr + 8u * slot, phase, p.status, aborted);
+            mbar_wait(full_addr + 8u * slot, phase, p.status, aborted, p.wait_limit_ns);
             const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk) + tid;
             if (c == 0) {
                 Mref = max8_scaled(*(const uint4*)(smem + (size_t)slot * kChunk));
@@ -521,7 +522,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, NW == 16 ? 1 : 3) row_ring_kerne
         const uint32_t sign2 = g > 0.f ? 0x80008000u : 0u;
         const float dy = g * r.one_m_py;
         for (int c = 0; c < chunks; ++c, dst += kChunk) {
-            if (!ra.resident) mbar_wait(full_addr + 8u * slot, phase, p.status, aborted);
+            if (!ra.resident) mbar_wait(full_addr + 8u * slot, phase, p.status, aborted, p.wait_limit_ns);
             const uint4* src = (const uint4*)(smem + (size_t)slot * kChunk) + tid;
             if (c < full_chunks && c != ychunk && g != 0.f) {
                 uint4 q[U];

@@ -16,8 +16,9 @@ __device__ __forceinline__ float reward_token(float lp_old, float lp_ref, float 
     return r;
 }
 
-__global__ void __launch_bounds__(256) kl_reward_kernel(const float* __restrict__ lp_old,
-                                                        const float* __restrict__ lp_ref,
+// lp_old and lp_ref carry no __restrict__: `out` may be one of them (each element is read before it is written,
+// by the same thread).
+__global__ void __launch_bounds__(256) kl_reward_kernel(const float* lp_old, const float* lp_ref,
                                                         const float* __restrict__ score,
                                                         const int* __restrict__ lengths, int B, int T,
                                                         float beta, float clip, float* out)
@@ -129,6 +130,107 @@ __global__ void __launch_bounds__(kGaeWarpsPerBlock * 32) reward_gae_kernel(cons
     gae_warp(rewards + off, values + off, n, T, gamma, lambda, adv + off, ret + off, lane);
 }
 
+// ---------------------------------------------------------------- optional: advantage whitening
+// (A - mean) / sqrt(var + eps) over the valid tokens of the whole batch, population variance, in two launches.
+// The first reduces sum and sum of squares in double precision in a fixed order (each block a contiguous range of
+// tokens with a fixed tree; the last block to finish adds the block partials in index order) and leaves mean and
+// 1/sqrt(var + eps) in the workspace; the second applies them.  No floating-point atomics: bit-stable.
+constexpr int kWhitenThreads = 256;
+constexpr int kWhitenMaxBlocks = 256;
+
+struct WhitenArgs {
+    const float* adv;
+    const int* lengths;
+    int B, T;
+    float eps;
+    float* out;
+    unsigned* ticket;           // workspace word 1, zero between calls
+    double* partials;           // workspace: [kWhitenMaxBlocks][2]
+    float* mean_rstd;           // workspace: 2 floats
+};
+
+__global__ void __launch_bounds__(kWhitenThreads) whiten_stats_kernel(WhitenArgs p)
+{
+    __shared__ double s_red[2][kWhitenThreads / 32];
+    __shared__ long long s_n[kWhitenThreads / 32];
+    __shared__ bool s_last;
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    const long long total = (long long)p.B * p.T;
+    const long long per_block = (total + gridDim.x - 1) / gridDim.x;
+    const long long begin = per_block * blockIdx.x, end = min(total, begin + per_block);
+    double s1 = 0.0, s2 = 0.0;
+    for (long long i = begin + threadIdx.x; i < end; i += blockDim.x) {
+        const int b = (int)(i / p.T), t = (int)(i % p.T);
+        if (t < clamp_len(__ldg(p.lengths + b), p.T)) {
+            const double a = (double)p.adv[i];
+            s1 += a;
+            s2 += a * a;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_red[0][warp] = s1; s_red[1][warp] = s2; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, c = 0.0;
+        for (int w = 0; w < kWhitenThreads / 32; ++w) { a += s_red[0][w]; c += s_red[1][w]; }
+        p.partials[2 * blockIdx.x] = a;
+        p.partials[2 * blockIdx.x + 1] = c;
+        __threadfence();
+        s_last = (atomicAdd(p.ticket, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    // the last block: number of valid tokens, then mean and 1/sqrt(var + eps)
+    long long n = 0;
+    for (int b = threadIdx.x; b < p.B; b += blockDim.x) n += clamp_len(__ldg(p.lengths + b), p.T);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+    if (lane == 0) s_n[warp] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        long long N = 0;
+        for (int w = 0; w < kWhitenThreads / 32; ++w) N += s_n[w];
+        double a = 0.0, c = 0.0;
+        for (unsigned k = 0; k < gridDim.x; ++k) {
+            a += ((volatile double*)p.partials)[2 * k];
+            c += ((volatile double*)p.partials)[2 * k + 1];
+        }
+        float mean = 0.f, rstd = 0.f;
+        if (N > 0) {
+            const double m = a / (double)N;
+            double var = c / (double)N - m * m;
+            if (var < 0.0) var = 0.0;
+            const double d = var + (double)p.eps;
+            mean = (float)m;
+            rstd = d > 0.0 ? (float)(1.0 / sqrt(d)) : 0.f;
+        }
+        p.mean_rstd[0] = mean;
+        p.mean_rstd[1] = rstd;
+        *p.ticket = 0u;
+    }
+}
+
+__global__ void __launch_bounds__(256) whiten_apply_kernel(WhitenArgs p)
+{
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    const float mean = p.mean_rstd[0], rstd = p.mean_rstd[1];
+    const long long total = (long long)p.B * p.T;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int b = (int)(i / p.T), t = (int)(i % p.T);
+        float w = 0.f;
+        if (t < clamp_len(__ldg(p.lengths + b), p.T)) w = (p.adv[i] - mean) * rstd;
+        p.out[i] = w;
+    }
+}
+
 // ---------------------------------------------------------------- step 4: finalisation
 // Value loss and dvalues per token, then both losses summed in a fixed order: each block reduces a
 // contiguous range of tokens with a fixed tree, the last block to finish (a ticket in the workspace)
@@ -220,7 +322,8 @@ __global__ void __launch_bounds__(kFinalThreads) ppo_finalize_kernel(FinalArgs p
 // (the row assignment is static); the last block to finish adds the block partials in index order.
 // The value-loss part: one thread's share of the block's slice; writes dvalues (and zeroes lp_new at
 // padding) and returns the thread's partial sum of loss terms.
-__device__ inline double value_loss_slice(const RowArgs& p, long long N, int tid, int nthreads)
+// zero_pad_terms: also writes 0 to the per-token policy loss terms (row_loss) of the padded tokens.
+__device__ inline double value_loss_slice(const RowArgs& p, long long N, int tid, int nthreads, bool zero_pad_terms = false)
 {
     const float scale_over_N = N > 0 ? p.grad_scale / (float)N : 0.f;
     const long long total = (long long)p.B * p.T;
@@ -236,8 +339,9 @@ __device__ inline double value_loss_slice(const RowArgs& p, long long N, int tid
             float e1 = (v - G) * (v - G), e2 = (vc - G) * (vc - G);
             if (e1 >= e2) { sum_vf += 0.5 * (double)e1; dv = (v - G) * scale_over_N; }
             else sum_vf += 0.5 * (double)e2;
-        } else if (p.out_lp_new) {
-            p.out_lp_new[i] = 0.f;
+        } else {
+            if (p.out_lp_new) p.out_lp_new[i] = 0.f;
+            if (zero_pad_terms) p.row_loss[i] = 0.f;
         }
         p.out_dvalues[i] = dv;
     }

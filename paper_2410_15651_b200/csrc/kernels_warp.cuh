@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
         Acc a = acc_empty();
         float zy = 0.f;
         for (int c = 0; c < row_chunks; ++c) {
-            mbar_wait(bar_addr + 8u * slot, (phases >> slot) & 1u, p.status, aborted);
+            mbar_wait(bar_addr + 8u * slot, (phases >> slot) & 1u, p.status, aborted, p.wait_limit_ns);
             phases ^= 1u << slot;
             const uint4* src = (const uint4*)(ring + (size_t)slot * kWarpChunk) + lane;
             if (c >= plain_begin && c < plain_end && c != ychunk) {
