@@ -283,7 +283,7 @@ def measure_workload(name, args, K, dev, rank, local_rank, world, with_e2e):
     # least DETAIL_MIN_MS have been timed (an event between two launches keeps the second from starting its
     # set-up under the tail of the first, so these steps are a little slower than the headline ones)
     exp_ms, loss_ms, detail_total = [], [], 0.0
-    while detail_total < DETAIL_MIN_MS or len(loss_ms) < DETAIL_MIN_LAUNCHES:
+    while detail_total < args.detail_ms or len(loss_ms) < min(DETAIL_MIN_LAUNCHES, K if args.detail_ms <= 0 else DETAIL_MIN_LAUNCHES):
         evs = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(K)]
         for i in range(K):
             path.step(evs[i])
@@ -557,6 +557,9 @@ def main():
                     help="override the number of sequences B of the workload (smaller cases for profiling)")
     ap.add_argument("--aux-steps", type=int, default=0,
                     help="steps per timed pass of the workloads after the first (default: about 0.5 s each)")
+    ap.add_argument("--detail-ms", type=float, default=DETAIL_MIN_MS,
+                    help="the event-timed pass repeats its steps until so many milliseconds have been timed "
+                         "(0: one pass of --steps steps, for runs under a profiler)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--in-place", action="store_true", help="dlogits overwrite the logits given to the loss call")
     ap.add_argument("--separate-calls", action="store_true",

@@ -104,6 +104,13 @@ int rlhf_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * the last poll (RLHF_OK if none) and clear them. */
 int rlhf_poll_status(void* workspace, void* stream);
 
+/* Self-test of the library's failure detection (the paper has no counterpart).  Every kernel that waits on a
+ * shared-memory barrier gives up after a bounded time, sets RLHF_ERR_TIMEOUT in the workspace and lets its block
+ * drain instead of hanging.  This call launches one warp that waits, with that same code, on a barrier at which
+ * nothing ever arrives, for at most limit_ns nanoseconds (0 < limit_ns <= 2e9), and returns.  Afterwards
+ * rlhf_poll_status reports RLHF_ERR_TIMEOUT once, and the workspace is usable as before.  Nothing faults. */
+int rlhf_selftest_bounded_wait(void* workspace, size_t workspace_bytes, unsigned long long limit_ns, void* stream);
+
 /*
  * Step 1 -- log-probability of the generated tokens (Section 2.1: the actor and reference
  * inferences that produce the experience).  For t < lengths[b], with z = logits[b,t,:], y = ids[b,t]:

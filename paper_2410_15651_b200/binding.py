@@ -29,6 +29,7 @@ SIGNATURES = {
     "rlhf_workspace_bytes": (_sz, [_int, _int]),
     "rlhf_workspace_init": (_int, [_vp, _sz, _vp]),
     "rlhf_poll_status": (_int, [_vp, _vp]),
+    "rlhf_selftest_bounded_wait": (_int, [_vp, _sz, ctypes.c_ulonglong, _vp]),
     "rlhf_gather_logprobs": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
     "rlhf_kl_reward": (_int, [_vp, _vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
     "rlhf_gae": (_int, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp, _vp]),
@@ -140,6 +141,12 @@ def workspace(B: int, T: int, device) -> torch.Tensor:
 def poll_status(ws: torch.Tensor) -> int:
     """Synchronise and return (then clear) the device-detected status flags."""
     return int(lib().rlhf_poll_status(ws.data_ptr(), _stream(ws)))
+
+
+def selftest_bounded_wait(ws: torch.Tensor, limit_ns: int) -> None:
+    """Launch the kernel whose only wait can never be satisfied; poll_status(ws) then reports the timeout flag."""
+    _check(lib().rlhf_selftest_bounded_wait(ws.data_ptr(), ws.numel(), int(limit_ns), _stream(ws)),
+           "rlhf_selftest_bounded_wait")
 
 
 def status_string(status: int) -> str:

@@ -183,7 +183,10 @@ int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 // most kRegVecsOnly vectors of a row, else in registers for its first kRegVecsTmem vectors and in tensor memory for
 // up to kTmemVecs more.  A block holds two buffers of its share of
 // a row; rows that do not fit twice are shared by a cluster of up to 4 blocks.
-constexpr int kCregWarps = 16;
+#ifndef RLHF_CREG_WARPS
+#define RLHF_CREG_WARPS 16
+#endif
+constexpr int kCregWarps = RLHF_CREG_WARPS;
 
 struct CregPlan {
     int cluster = 0;            // blocks per cluster, 1..4; 0 = the kernel does not apply
@@ -415,6 +418,14 @@ int rlhf_poll_status(void* workspace, void* stream)
         RLHF_CUDA(cudaStreamSynchronize(s));
     }
     return (int)flags;
+}
+
+int rlhf_selftest_bounded_wait(void* workspace, size_t workspace_bytes, unsigned long long limit_ns, void* stream)
+{
+    if (int e = check_workspace(workspace, workspace_bytes, kRowLossOffset)) return e;
+    if (limit_ns == 0 || limit_ns > kWaitLimitNs) return RLHF_ERR_SCALAR;
+    RLHF_CUDA(launch_kernel(bounded_wait_selftest_kernel, 1, 32, 0, (cudaStream_t)stream, (unsigned*)workspace, limit_ns));
+    return launch_check("bounded_wait_selftest_kernel");
 }
 
 int rlhf_gather_logprobs(const void* logits, long long stride_b, long long stride_t,

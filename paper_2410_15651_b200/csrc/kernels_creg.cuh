@@ -41,7 +41,10 @@
 
 namespace rlhf {
 
-constexpr int kRegVecsOnly = 8;        // vectors per consumer thread when the registers hold all of a thread's exponentials
+#ifndef RLHF_CREG_REGVECS_ONLY
+#define RLHF_CREG_REGVECS_ONLY 8
+#endif
+constexpr int kRegVecsOnly = RLHF_CREG_REGVECS_ONLY;        // vectors per consumer thread when the registers hold all of a thread's exponentials
 constexpr int kRegVecsTmem = 4;        // vectors per consumer thread kept in registers when the rest goes to tensor memory
 constexpr int kTmemVecs = 16;          // at most so many vectors per consumer thread in tensor memory
 constexpr int kCregZeroBytes = 16384;  // zeroed buffer that feeds the bulk zero-fill of padded rows
@@ -79,7 +82,7 @@ inline unsigned creg_tmem_cols(unsigned slice_vecs, int consumer_warps)
     const unsigned per_round = (unsigned)consumer_warps * 32;
     const unsigned nj = (slice_vecs + per_round - 1) / per_round;
     if (nj <= (unsigned)kRegVecsOnly) return 0;
-    const unsigned need = (nj - kRegVecsTmem) * 8 * ((unsigned)consumer_warps / 4);
+    const unsigned need = (nj - kRegVecsTmem) * 8 * (((unsigned)consumer_warps + 3) / 4);
     unsigned cols = 32;
     while (cols < need) cols *= 2;
     return cols;
@@ -197,7 +200,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ long long s_cnt[33];
     __shared__ float2 s_part[2][32];
-    __shared__ __align__(16) float s_sum[2][NW];
+    __shared__ __align__(16) float s_sum[2][(NW + 3) / 4 * 4];
     __shared__ LabelInfo s_lab[2];
     __shared__ RowInfo s_row[kCregMaxBufs];
     __shared__ double s_dbl[32];

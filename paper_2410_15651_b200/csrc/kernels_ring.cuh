@@ -108,6 +108,23 @@ __device__ __forceinline__ void store_v4(void* p, const uint4& q)
                  : "memory");
 }
 
+// One block of one warp that waits, with the bounded wait every pipelined kernel of the library uses, on a
+// shared-memory barrier at which nobody ever arrives: the wait runs out after `limit_ns`, the status word gets
+// RLHF_ERR_TIMEOUT and the kernel returns.  It exists so that the give-up path can be exercised without a fault.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(unsigned* status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long s_bar;
+    const uint32_t bar = smem_u32(&s_bar);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    bool aborted = false;
+    mbar_wait(bar, 0u, status, aborted, limit_ns);
+    // (aborted is true here on every thread; nothing else to release)
+}
+
 // ---------------------------------------------------------------- 8 logits at a time
 __device__ __forceinline__ void unpack8(const uint4& q, float (&z)[8])
 {
@@ -277,9 +294,10 @@ __device__ __forceinline__ bool consumer_barrier_or(bool flag)
 template <int NW>
 __device__ __forceinline__ float sum_warp_sums(const float* s_sum)
 {
-    float v[NW];
+    // (the array is read in whole float4s: it holds a multiple of 4 floats, of which the first NW are used)
+    float v[(NW + 3) / 4 * 4];
 #pragma unroll
-    for (int w4 = 0; w4 < NW / 4; ++w4) {
+    for (int w4 = 0; w4 < (NW + 3) / 4; ++w4) {
         const float4 t4 = ((const float4*)s_sum)[w4];
         v[4 * w4] = t4.x; v[4 * w4 + 1] = t4.y; v[4 * w4 + 2] = t4.z; v[4 * w4 + 3] = t4.w;
     }

@@ -90,6 +90,23 @@ def test_host_side_argument_checks(lib):
     assert s4(dst=7) == 4 and s4(dsb=24) == 4                # rows too close / sequences overlapping
     assert s4(dl=p, dsb=64) == 4                             # in place needs equal strides
     assert s4(wsn=100) == 5
+    # B*T above 2^29 is refused (the log-prob kernel walks up to 2*B*T rows with 32-bit indices)
+    big = lib.rlhf_workspace_bytes(1 << 15, 1 << 14)
+    assert s1(B=1 << 15, T=1 << 14, wsn=big - 256) == 5      # exactly 2^29 passes the shape check (the workspace is checked next)
+    assert s1(B=(1 << 15) + 1, T=1 << 14) == 2
+    assert s4(B=(1 << 15) + 1, T=1 << 14) == 2
+    assert lib.rlhf_kl_reward(p, p, p, p, (1 << 15) + 1, 1 << 14, 0.1, 5.0, p, None) == 2
+    # whitening
+    assert lib.rlhf_whiten_advantages(None, p, 2, 4, 1e-8, p, p, ws_n, None) == 1
+    assert lib.rlhf_whiten_advantages(p, p, 2, 4, -1.0, p, p, ws_n, None) == 6
+    assert lib.rlhf_whiten_advantages(p, p, 2, 4, float("inf"), p, p, ws_n, None) == 6
+    assert lib.rlhf_whiten_advantages(p, p, 2, 4, 1e-8, p, p, 8, None) == 5
+    assert lib.rlhf_whiten_advantages(p, p, 0, 4, 1e-8, p, p, ws_n, None) == 2
+    # bounded-wait self-test: limit must be positive and at most 2 s
+    assert lib.rlhf_selftest_bounded_wait(None, ws_n, 1000, None) == 1
+    assert lib.rlhf_selftest_bounded_wait(p, ws_n, 0, None) == 6
+    assert lib.rlhf_selftest_bounded_wait(p, ws_n, 3 * 10 ** 9, None) == 6
+    assert lib.rlhf_selftest_bounded_wait(p, 100, 1000, None) == 5
 
 
 def test_binding_refuses_cpu_tensors():

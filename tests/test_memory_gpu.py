@@ -49,6 +49,11 @@ def test_library_calls_allocate_nothing():
 
 
 def test_in_place_gradient_needs_no_logits_sized_buffer_and_empty_cache_releases_the_rest():
+    # start from an empty allocator cache, so that this test's tensors do not share segments with blocks that
+    # earlier tests left cached (a segment goes back to the driver only when all of it is free)
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     w = inputs.scaled(inputs.WORKLOADS["llama2"], B=4, T=128)
     batch, ws, exp = _setup(w)
     logits_bytes = batch["actor"].numel() * 2

@@ -4,8 +4,11 @@ configuration the benchmark times.
 
 Every O(B*T) output (log-probs of all rows for actor and reference, rewards, advantages, returns,
 dvalues, both losses) is compared in full: the oracle computes all of them.  The bf16 logits
-gradient is compared element by element on a sample of rows (valid, padded, zero-gradient, first
-and last), and checked on every row through properties that need no oracle row.
+gradient is compared element by element on every row for the OPT- and Llama-2-shaped workloads
+(out of place), and for the others on a sample of rows (valid, padded, zero-gradient, first and
+last, and for the large-vocabulary workload, whose rows are dealt statically to clusters of blocks,
+the first and the last 64 valid rows, which covers every cluster at the start and at the end of
+its work); every row is also checked through properties that need no oracle row.
 """
 import numpy as np
 import pytest
@@ -26,8 +29,12 @@ def test_full_size(oracle, name, in_place):
     batch = inputs.make_batch(w, device=DEV)
     run = OracleRun(oracle, w, batch)
     rows = sample_rows(run, 48, seed=w.seed)
+    if name == "large_vocab":
+        flat_valid = np.flatnonzero(run.valid.reshape(-1))
+        rows = np.unique(np.concatenate([rows, flat_valid[:64], flat_valid[-64:]]))
+    every_row = name in ("opt", "llama2") and not in_place
     out, rep = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"],
-                         in_place=in_place, sample_rows=rows)
+                         in_place=in_place, sample_rows=rows, all_rows=every_row)
     dlogits_properties(run, out, batch["ids"], batch["actor"])
     if not in_place:
         _experience_both_ways(w, batch, batch["actor"], batch["ref"], batch["ids"])
