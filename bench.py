@@ -250,6 +250,9 @@ def measure_workload(name, args, K, dev, rank, local_rank, world, with_e2e):
     if args.sequences > 0:
         w = inputs.scaled(w, B=args.sequences)
     batch = inputs.make_batch(w, device=dev)
+    if args.logits_dtype == "fp16":
+        batch["actor"] = batch["actor"].to(torch.float16)
+        batch["ref"] = batch["ref"].to(torch.float16)
     path = Path(w, batch, dev, fused=not args.separate_calls, in_place=args.in_place, global_mean=args.global_mean)
     B, T, V = w.B, w.T, w.V
     n_valid = path.N
@@ -422,7 +425,7 @@ def run_ours(args):
         "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{head['name']}: B={B} T={T} V={V} bf16 logits, {head['n_valid']} response tokens per GPU",
+        "config": {"workload": f"{head['name']}: B={B} T={T} V={V} {args.logits_dtype} logits, {head['n_valid']} response tokens per GPU",
                    "also_timed": [n for n in names[1:]],
                    "l2": "inputs larger than L2 (%.2f GB touched per step)" % (head["step_bytes"] / 1e9),
                    "multi_gpu": ("one batch shard per rank; token counts all-reduced (NCCL) before the loss call, "
@@ -560,6 +563,8 @@ def main():
     ap.add_argument("--detail-ms", type=float, default=DETAIL_MIN_MS,
                     help="the event-timed pass repeats its steps until so many milliseconds have been timed "
                          "(0: one pass of --steps steps, for runs under a profiler)")
+    ap.add_argument("--logits-dtype", default="bf16", choices=["bf16", "fp16"],
+                    help="element type of the logits and of their gradient")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--in-place", action="store_true", help="dlogits overwrite the logits given to the loss call")
     ap.add_argument("--separate-calls", action="store_true",

@@ -14,6 +14,7 @@
  *   rlhf_ppo_loss_fwd_bwd   clipped policy and value loss, gradient w.r.t. the logits and values
  *   rlhf_experience         the first three together (both log-prob passes in one kernel, reward + GAE in another)
  *   rlhf_whiten_advantages  optional masked whitening of the advantages between steps 3 and 4
+ *   rlhf_ppo_stats          monitors of the policy step: approximate KL to the old policy, clip fraction
  *
  * The paper gives these quantities in prose only; the formulas are the standard definitions and
  * are written out beside each function.
@@ -28,7 +29,7 @@
  *    on `stream` (a cudaStream_t passed as void*, NULL = the default stream) and never
  *    synchronise it (rlhf_poll_status excepted).
  *  - [B,T] arrays are fp32 (ids int64, lengths int32), row-major, T contiguous.
- *  - Logits are bf16, addressed as base[b*stride_b + t*stride_t + v], strides in ELEMENTS,
+ *  - Logits are bf16 (binary16 through the *_ex entry points), addressed as base[b*stride_b + t*stride_t + v], strides in ELEMENTS,
  *    stride_t >= V.  For a full-sequence tensor [B,P+T,V] whose row P-1+t predicts response
  *    token t, pass base + (P-1)*V, stride_b = (P+T)*V, stride_t = V, and ids = input_ids + P with
  *    ids_stride_b = P+T.  Rows whose start address and byte length are multiples of 16 take the
@@ -72,6 +73,17 @@ typedef enum {
     RLHF_ERR_LENGTH_RANGE = 32, /* a length outside [0,T] (clamped) */
     RLHF_ERR_TIMEOUT = 64       /* an internal bounded wait ran out; outputs of this call are invalid */
 } rlhf_status_t;
+
+/* Element type of a logits tensor (and of the gradient written for it): the two 16-bit floating-point
+ * types the paper's model families are run in (Section 3, "Workload and Setting").  The entry points
+ * without a type argument take bf16; the *_ex ones take either.  Widening is exact; the gradient is
+ * rounded to nearest even in the same type.  binary16 cannot hold magnitudes above 65504: a gradient
+ * entry is at most |g| = grad_scale * |A| * rho / N in magnitude, so keep grad_scale such that this stays
+ * below that bound (with grad_scale = 1 it always does), else the entry becomes +-inf. */
+typedef enum {
+    RLHF_BF16 = 0,
+    RLHF_F16 = 1
+} rlhf_dtype_t;
 
 /* Human-readable name of a status (static storage; flags are joined with '|'). Host, never NULL. */
 const char* rlhf_status_string(int status);
@@ -126,6 +138,20 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
                          const long long* ids, long long ids_stride_b, const int* lengths,
                          int B, int T, int V, float* out_logprobs,
                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Step 1 with options: the element type of the logits (an rlhf_dtype_t) and, if out_entropy is not NULL, the
+ * entropy of the softmax of every valid row,
+ *     out_entropy[b,t] = - sum_v p_v log p_v,   p_v = exp(z_v - log sum_u exp(z_u))      (nats),
+ * 0 at padded positions; a deleted entry (z_v = -inf) adds 0.  The entropy costs one more multiply-add per logit in
+ * the same streaming pass, no extra memory traffic.  At a token whose id is out of range the log-prob is 0 (and
+ * the status flag is set) but the entropy, which does not depend on the id, is still that of the row.
+ * Everything else as rlhf_gather_logprobs.   RLHF_ERR_SCALAR for an unknown logits_dtype.
+ */
+int rlhf_gather_logprobs_ex(const void* logits, int logits_dtype, long long stride_b, long long stride_t,
+                            const long long* ids, long long ids_stride_b, const int* lengths,
+                            int B, int T, int V, float* out_logprobs, float* out_entropy,
+                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Step 2 -- per-token reward (Section 2.1: the reference model prevents reward divergence, the
@@ -192,6 +218,16 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
                     float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
                     float* out_returns, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Steps 1-3 together with options: the element type of both logits tensors, and (if not NULL) the entropy of
+ * the actor's rows as in rlhf_gather_logprobs_ex.  Everything else as rlhf_experience. */
+int rlhf_experience_ex(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
+                       const void* ref_logits, long long ref_stride_b, long long ref_stride_t, int logits_dtype,
+                       const long long* ids, long long ids_stride_b, const int* lengths,
+                       const float* score, const float* values_old, const float* lp_old,
+                       int B, int T, int V, float beta_kl, float reward_clip, float gamma, float lambda,
+                       float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
+                       float* out_returns, float* out_entropy, void* workspace, size_t workspace_bytes, void* stream);
+
 /*
  * Step 4 -- clipped PPO losses and their gradients (Section 2.1: the actor is trained to maximise
  * reward while limiting policy deviation, the critic is trained on the returns).  For each valid
@@ -225,6 +261,34 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
                           void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
                           float* out_dvalues, float* out_lp_new,
                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 4 with the element type of logits and out_dlogits (an rlhf_dtype_t; both tensors have the same type).
+ * Everything else as rlhf_ppo_loss_fwd_bwd.  RLHF_ERR_SCALAR for an unknown logits_dtype. */
+int rlhf_ppo_loss_fwd_bwd_ex(const void* logits, int logits_dtype, long long stride_b, long long stride_t,
+                             const long long* ids, long long ids_stride_b, const int* lengths,
+                             const float* lp_old, const float* adv, const float* values_new,
+                             const float* values_old, const float* returns,
+                             int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
+                             float* out_loss_pg, float* out_loss_vf,
+                             void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                             float* out_dvalues, float* out_lp_new,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Monitors of the policy step (Section 2.1: the actor is trained "while minimizing policy deviation"; these two
+ * numbers are how that deviation is watched).  From the log-probs that step 4 returns in out_lp_new:
+ *     rho = exp(lp_new - lp_old)
+ *     out_stats[0] = approx_kl = (1/N) sum ((rho - 1) - log rho)          (non-negative, 0 on policy)
+ *     out_stats[1] = clip_frac = (1/N) #{ -A*clamp(rho, 1-clip_eps, 1+clip_eps) > -A*rho }
+ * over the valid tokens; both 0 if N = 0.  clip_frac is the share of tokens to which step 4 gives a zero
+ * gradient; a token whose ratio sits on the edge of the interval to within float32 rounding may be counted on
+ * either side.  Sums in double precision in a fixed order.
+ *   lp_new, lp_old, adv   fp32 [B,T]; lengths int32 [B]                 read
+ *   out_stats             fp32 [2] (device)                              written
+ *   clip_eps in (0,1).   workspace as for step 1.
+ */
+int rlhf_ppo_stats(const float* lp_new, const float* lp_old, const float* adv, const int* lengths, int B, int T,
+                   float clip_eps, float* out_stats, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Step 4 for callers that cannot provide a workspace.  (The paper has no counterpart to this

@@ -31,9 +31,16 @@ SIGNATURES = {
     "rlhf_poll_status": (_int, [_vp, _vp]),
     "rlhf_selftest_bounded_wait": (_int, [_vp, _sz, ctypes.c_ulonglong, _vp]),
     "rlhf_gather_logprobs": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
+    "rlhf_gather_logprobs_ex": (_int, [_vp, _int, _i64, _i64, _vp, _i64, _vp, _int, _int, _int, _vp, _vp, _vp, _sz, _vp]),
+    "rlhf_experience_ex": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _int, _vp, _i64, _vp, _vp, _vp, _vp,
+                                  _int, _int, _int, _f32, _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "rlhf_ppo_loss_fwd_bwd_ex": (_int, [_vp, _int, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
+                                        _int, _int, _int, _f32, _f32, _f32, _vp, _vp,
+                                        _vp, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
     "rlhf_kl_reward": (_int, [_vp, _vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
     "rlhf_gae": (_int, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp, _vp]),
     "rlhf_whiten_advantages": (_int, [_vp, _vp, _int, _int, _f32, _vp, _vp, _sz, _vp]),
+    "rlhf_ppo_stats": (_int, [_vp, _vp, _vp, _vp, _int, _int, _f32, _vp, _vp, _sz, _vp]),
     "rlhf_experience": (_int, [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp,
                                _int, _int, _int, _f32, _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "rlhf_ppo_loss_fwd_bwd": (_int, [_vp, _i64, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -106,8 +113,14 @@ def _bt(t: torch.Tensor, B: int, T: int, what: str) -> torch.Tensor:
     return t
 
 
+DTYPES = {torch.bfloat16: 0, torch.float16: 1}        # rlhf_dtype_t
+
+
 def _logits(t: torch.Tensor, what: str) -> Tuple[int, int, int, int, int]:
-    _dev(t, torch.bfloat16, what)
+    if not t.is_cuda:
+        raise ValueError(f"{what} must be a CUDA tensor (the library has no CPU path)")
+    if t.dtype not in DTYPES:
+        raise TypeError(f"{what} must be bfloat16 or float16, got {t.dtype}")
     if t.dim() != 3 or (t.shape[2] > 1 and t.stride(2) != 1):
         raise ValueError(f"{what} must be [B,T,V] with a contiguous vocabulary axis")
     return t.shape[0], t.shape[1], t.shape[2], t.stride(0), t.stride(1)
@@ -154,16 +167,24 @@ def status_string(status: int) -> str:
 
 
 def gather_logprobs(logits: torch.Tensor, ids: torch.Tensor, lengths: torch.Tensor,
-                    ws: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                    ws: torch.Tensor, out: Optional[torch.Tensor] = None,
+                    out_entropy: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """rlhf_gather_logprobs for bf16 logits without an entropy output, else rlhf_gather_logprobs_ex."""
     B, T, V, sb, st = _logits(logits, "logits")
     isb = _ids(ids, B, T)
     _lengths(lengths, B)
     if out is None:
         out = torch.empty((B, T), dtype=torch.float32, device=logits.device)
     _bt(out, B, T, "out")
-    _check(lib().rlhf_gather_logprobs(logits.data_ptr(), sb, st, ids.data_ptr(), isb, lengths.data_ptr(),
-                                      B, T, V, out.data_ptr(), ws.data_ptr(), ws.numel(), _stream(logits)),
-           "rlhf_gather_logprobs")
+    if logits.dtype == torch.bfloat16 and out_entropy is None:
+        _check(lib().rlhf_gather_logprobs(logits.data_ptr(), sb, st, ids.data_ptr(), isb, lengths.data_ptr(),
+                                          B, T, V, out.data_ptr(), ws.data_ptr(), ws.numel(), _stream(logits)),
+               "rlhf_gather_logprobs")
+        return out
+    ent_ptr = _bt(out_entropy, B, T, "out_entropy").data_ptr() if out_entropy is not None else None
+    _check(lib().rlhf_gather_logprobs_ex(logits.data_ptr(), DTYPES[logits.dtype], sb, st, ids.data_ptr(), isb,
+                                         lengths.data_ptr(), B, T, V, out.data_ptr(), ent_ptr,
+                                         ws.data_ptr(), ws.numel(), _stream(logits)), "rlhf_gather_logprobs_ex")
     return out
 
 
@@ -215,6 +236,22 @@ def whiten_advantages(adv: torch.Tensor, lengths: torch.Tensor, eps: float, ws: 
     return out
 
 
+def ppo_stats(lp_new: torch.Tensor, lp_old: torch.Tensor, adv: torch.Tensor, lengths: torch.Tensor,
+              clip_eps: float, ws: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """[approx_kl, clip_frac] of the policy step, as a device tensor of two floats."""
+    B, T = lp_new.shape
+    for name, t in (("lp_new", lp_new), ("lp_old", lp_old), ("adv", adv)):
+        _bt(t, B, T, name)
+    _lengths(lengths, B)
+    if out is None:
+        out = torch.empty(2, dtype=torch.float32, device=lp_new.device)
+    _dev(out, torch.float32, "out")
+    _check(lib().rlhf_ppo_stats(lp_new.data_ptr(), lp_old.data_ptr(), adv.data_ptr(), lengths.data_ptr(), B, T,
+                                clip_eps, out.data_ptr(), ws.data_ptr(), ws.numel(), _stream(lp_new)),
+           "rlhf_ppo_stats")
+    return out
+
+
 class Experience:
     """Buffers written by experience(); reusable from call to call."""
 
@@ -226,7 +263,8 @@ class Experience:
 def experience(actor_logits: torch.Tensor, ref_logits: torch.Tensor, ids: torch.Tensor, lengths: torch.Tensor,
                score: torch.Tensor, values_old: torch.Tensor, beta_kl: float, reward_clip: float,
                gamma: float, lam: float, ws: torch.Tensor, out: Optional[Experience] = None,
-               lp_old: Optional[torch.Tensor] = None) -> Experience:
+               lp_old: Optional[torch.Tensor] = None, out_entropy: Optional[torch.Tensor] = None) -> Experience:
+    """rlhf_experience for bf16 logits without an entropy output, else rlhf_experience_ex."""
     B, T, V, asb, ast = _logits(actor_logits, "actor_logits")
     rB, rT, rV, rsb, rst = _logits(ref_logits, "ref_logits")
     if (rB, rT, rV) != (B, T, V):
@@ -242,6 +280,17 @@ def experience(actor_logits: torch.Tensor, ref_logits: torch.Tensor, ids: torch.
     for name in ("lp_actor", "lp_ref", "rewards", "adv", "returns"):
         _bt(getattr(out, name), B, T, "out." + name)
     lp_old_ptr = _bt(lp_old, B, T, "lp_old").data_ptr() if lp_old is not None else None
+    if actor_logits.dtype != ref_logits.dtype:
+        raise TypeError("actor and reference logits must have the same element type")
+    if actor_logits.dtype != torch.bfloat16 or out_entropy is not None:
+        ent_ptr = _bt(out_entropy, B, T, "out_entropy").data_ptr() if out_entropy is not None else None
+        _check(lib().rlhf_experience_ex(
+            actor_logits.data_ptr(), asb, ast, ref_logits.data_ptr(), rsb, rst, DTYPES[actor_logits.dtype],
+            ids.data_ptr(), isb, lengths.data_ptr(), score.data_ptr(), values_old.data_ptr(), lp_old_ptr, B, T, V,
+            beta_kl, reward_clip, gamma, lam, out.lp_actor.data_ptr(), out.lp_ref.data_ptr(),
+            out.rewards.data_ptr(), out.adv.data_ptr(), out.returns.data_ptr(), ent_ptr,
+            ws.data_ptr(), ws.numel(), _stream(actor_logits)), "rlhf_experience_ex")
+        return out
     _check(lib().rlhf_experience(
         actor_logits.data_ptr(), asb, ast, ref_logits.data_ptr(), rsb, rst, ids.data_ptr(), isb,
         lengths.data_ptr(), score.data_ptr(), values_old.data_ptr(), lp_old_ptr, B, T, V,
@@ -258,7 +307,7 @@ class PPOOutputs:
         B, T = logits.shape[0], logits.shape[1]
         dev = logits.device
         self.loss = torch.empty(2, dtype=torch.float32, device=dev)       # [loss_pg, loss_vf]
-        self.dlogits = logits if in_place else torch.empty(logits.shape, dtype=torch.bfloat16, device=dev)
+        self.dlogits = logits if in_place else torch.empty(logits.shape, dtype=logits.dtype, device=dev)
         self.dvalues = torch.empty((B, T), dtype=torch.float32, device=dev)
         self.lp_new = torch.empty((B, T), dtype=torch.float32, device=dev) if want_lp_new else None
 
@@ -284,6 +333,17 @@ def ppo_loss_fwd_bwd(logits: torch.Tensor, ids: torch.Tensor, lengths: torch.Ten
     if out.lp_new is not None:
         lp_new_ptr = _bt(out.lp_new, B, T, "out.lp_new").data_ptr()
     loss = _dev(out.loss, torch.float32, "out.loss")
+    if out.dlogits.dtype != logits.dtype:
+        raise TypeError("out.dlogits must have the element type of logits")
+    if logits.dtype != torch.bfloat16:
+        _check(lib().rlhf_ppo_loss_fwd_bwd_ex(
+            logits.data_ptr(), DTYPES[logits.dtype], sb, st, ids.data_ptr(), isb, lengths.data_ptr(),
+            lp_old.data_ptr(), adv.data_ptr(), values_new.data_ptr(), values_old.data_ptr(), returns.data_ptr(),
+            B, T, V, clip_eps, value_clip, grad_scale,
+            loss.data_ptr(), loss.data_ptr() + 4,
+            out.dlogits.data_ptr(), dsb, dst, out.dvalues.data_ptr(), lp_new_ptr,
+            ws.data_ptr(), ws.numel(), _stream(logits)), "rlhf_ppo_loss_fwd_bwd_ex")
+        return out
     _check(lib().rlhf_ppo_loss_fwd_bwd(
         logits.data_ptr(), sb, st, ids.data_ptr(), isb, lengths.data_ptr(),
         lp_old.data_ptr(), adv.data_ptr(), values_new.data_ptr(), values_old.data_ptr(), returns.data_ptr(),
@@ -304,6 +364,8 @@ def ppo_loss_fwd_bwd_noalloc(logits: torch.Tensor, ids: torch.Tensor, lengths: t
     not overlap).  `out` must be given (this wrapper allocates nothing either); `device_status`,
     if given, is an int32 CUDA tensor of one element that receives the device-detected flags."""
     B, T, V, sb, st = _logits(logits, "logits")
+    if logits.dtype != torch.bfloat16 or out.dlogits.dtype != torch.bfloat16:
+        raise TypeError("rlhf_ppo_loss_fwd_bwd_noalloc takes bf16 logits")
     isb = _ids(ids, B, T)
     _lengths(lengths, B)
     for name, t in (("lp_old", lp_old), ("adv", adv), ("values_new", values_new),

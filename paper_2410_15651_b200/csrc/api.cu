@@ -142,18 +142,29 @@ int launch_ring_as(const RingArgs& ra, const RingPlan& pl, int grid, cudaStream_
 
 constexpr int kLogprobWarps = 24;
 
-template <bool kDual, bool kAny = false>
-int launch_warp_logprob(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream_t s)
+template <bool kDual, bool kAny, bool kF16, bool kEnt>
+int launch_warp_logprob_as(const WarpArgs& wa_in, const DeviceInfo& dev, cudaStream_t s)
 {
     WarpArgs wa = wa_in;
     wa.row_bytes = 2u * (unsigned)wa.row.V;
     const size_t smem = warp_kernel_smem_bytes(kLogprobWarps);
     const long long rows = (long long)wa.row.B * wa.row.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps, kDual, kAny>,
+    RLHF_CUDA(cudaFuncSetAttribute(logprob_warp_kernel<kLogprobWarps, kDual, kAny, kF16, kEnt>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    RLHF_CUDA(launch_kernel(logprob_warp_kernel<kLogprobWarps, kDual, kAny>, grid, kLogprobWarps * 32, smem, s, wa));
+    RLHF_CUDA(launch_kernel(logprob_warp_kernel<kLogprobWarps, kDual, kAny, kF16, kEnt>, grid, kLogprobWarps * 32, smem, s, wa));
     return RLHF_OK;
+}
+
+// f16: the logits are IEEE binary16; the entropy variant is taken when wa.out_entropy is set.
+template <bool kDual, bool kAny>
+int launch_warp_logprob(const WarpArgs& wa, bool f16, const DeviceInfo& dev, cudaStream_t s)
+{
+    const bool ent = wa.out_entropy != nullptr;
+    if (f16) return ent ? launch_warp_logprob_as<kDual, kAny, true, true>(wa, dev, s)
+                        : launch_warp_logprob_as<kDual, kAny, true, false>(wa, dev, s);
+    return ent ? launch_warp_logprob_as<kDual, kAny, false, true>(wa, dev, s)
+               : launch_warp_logprob_as<kDual, kAny, false, false>(wa, dev, s);
 }
 
 constexpr int kDbufWarps = 16;
@@ -164,7 +175,7 @@ bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev, bool any_alignment 
     return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes, any_alignment) + 1280 <= (size_t)dev.max_smem_optin;
 }
 
-template <bool kAny>
+template <bool kAny, bool kF16>
 int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
 {
     DbufArgs da{};
@@ -174,8 +185,8 @@ int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
     const size_t smem = dbuf_smem_bytes(da.row_bytes, kAny);
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps, kAny>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    RLHF_CUDA(launch_kernel(loss_dbuf_kernel<kDbufWarps, kAny>, grid, kDbufWarps * 32 + 32, smem, s, da));
+    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps, kAny, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    RLHF_CUDA(launch_kernel(loss_dbuf_kernel<kDbufWarps, kAny, kF16>, grid, kDbufWarps * 32 + 32, smem, s, da));
     return RLHF_OK;
 }
 
@@ -220,7 +231,7 @@ CregPlan plan_creg(unsigned row_bytes, const DeviceInfo& dev)
 
 // Clusters of the kernel that the device holds at once (one block per SM); looked up once per device and
 // cluster size.  It only sizes the persistent grid: a larger grid would still be correct.
-template <int NW, int C, bool kTmem>
+template <int NW, int C, bool kTmem, bool kF16>
 int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
 {
     if (C == 1) { out = dev.sm_count; return RLHF_OK; }
@@ -234,7 +245,7 @@ int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attr[2];
         fill_launch_config(cfg, attr, dev.sm_count / C * C, NW * 32 + 32, pl.smem_bytes, C, nullptr);
-        RLHF_CUDA(cudaOccupancyMaxActiveClusters(&n, loss_creg_kernel<NW, C, kTmem>, &cfg));
+        RLHF_CUDA(cudaOccupancyMaxActiveClusters(&n, loss_creg_kernel<NW, C, kTmem, kF16>, &cfg));
         if (n < 1) n = 1;
         if (d < 0 || d >= 64) { out = n; return RLHF_OK; }
         cached[d] = n;
@@ -243,7 +254,7 @@ int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
     return RLHF_OK;
 }
 
-template <int NW, int C, bool kTmem>
+template <int NW, int C, bool kTmem, bool kF16>
 int launch_creg(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cudaStream_t s)
 {
     CregArgs ca{};
@@ -254,37 +265,48 @@ int launch_creg(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cud
     ca.tmem_cols = pl.tmem_cols;
     ca.n_buf = pl.n_buf;
     ca.row_counter = (unsigned*)((char*)a.status + 16);
-    RLHF_CUDA(cudaFuncSetAttribute(loss_creg_kernel<NW, C, kTmem>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RLHF_CUDA(cudaFuncSetAttribute(loss_creg_kernel<NW, C, kTmem, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)pl.smem_bytes));
     int clusters = 0;
-    if (int e = creg_resident_clusters<NW, C, kTmem>(pl, dev, clusters)) return e;
+    if (int e = creg_resident_clusters<NW, C, kTmem, kF16>(pl, dev, clusters)) return e;
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, clusters) * C;
-    RLHF_CUDA(launch_kernel_cluster(loss_creg_kernel<NW, C, kTmem>, grid, NW * 32 + 32, pl.smem_bytes, C, s, ca));
+    RLHF_CUDA(launch_kernel_cluster(loss_creg_kernel<NW, C, kTmem, kF16>, grid, NW * 32 + 32, pl.smem_bytes, C, s, ca));
     return RLHF_OK;
 }
 
-template <int NW, bool kTmem>
+template <int NW, bool kTmem, bool kF16>
 int launch_creg_cluster(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cudaStream_t s)
 {
     switch (pl.cluster) {
-        case 1: return launch_creg<NW, 1, kTmem>(a, pl, dev, s);
-        case 2: return launch_creg<NW, 2, kTmem>(a, pl, dev, s);
-        case 3: return launch_creg<NW, 3, kTmem>(a, pl, dev, s);
-        default: return launch_creg<NW, 4, kTmem>(a, pl, dev, s);
+        case 1: return launch_creg<NW, 1, kTmem, kF16>(a, pl, dev, s);
+        case 2: return launch_creg<NW, 2, kTmem, kF16>(a, pl, dev, s);
+        case 3: return launch_creg<NW, 3, kTmem, kF16>(a, pl, dev, s);
+        default: return launch_creg<NW, 4, kTmem, kF16>(a, pl, dev, s);
     }
 }
 
 // The loss row kernel for 16-byte aligned rows: exponentials in registers where the row (or its share in a
 // cluster) fits, else two resident rows, else the chunk ring.
-int launch_loss_rows(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
+// The fast loss kernels for 16-byte aligned rows of this length (binary16 rows: the on-chip-exponentials kernel
+// only; the chunk ring is a bf16 kernel).
+bool fast_loss_rows_apply(int V, bool f16, const DeviceInfo& dev)
+{
+    return !f16 || plan_creg(2u * (unsigned)V, dev).cluster > 0;
+}
+
+int launch_loss_rows(const RowArgs& a, bool f16, const DeviceInfo& dev, cudaStream_t s)
 {
     const unsigned row_bytes = 2u * (unsigned)a.V;
     const CregPlan cp = plan_creg(row_bytes, dev);
-    if (cp.cluster > 0)
-        return cp.tmem_cols != 0 ? launch_creg_cluster<kCregWarps, true>(a, cp, dev, s)
-                                 : launch_creg_cluster<kCregWarps, false>(a, cp, dev, s);
-    if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false>(a, dev, s);
+    if (cp.cluster > 0) {
+        if (f16)
+            return cp.tmem_cols != 0 ? launch_creg_cluster<kCregWarps, true, true>(a, cp, dev, s)
+                                     : launch_creg_cluster<kCregWarps, false, true>(a, cp, dev, s);
+        return cp.tmem_cols != 0 ? launch_creg_cluster<kCregWarps, true, false>(a, cp, dev, s)
+                                 : launch_creg_cluster<kCregWarps, false, false>(a, cp, dev, s);
+    }
+    if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false, false>(a, dev, s);
     const RingPlan pl = plan_ring(row_bytes, dev.smem_per_sm, dev.max_smem_optin);
     RingArgs ra{};
     ra.row = a;
@@ -428,17 +450,20 @@ int rlhf_selftest_bounded_wait(void* workspace, size_t workspace_bytes, unsigned
     return launch_check("bounded_wait_selftest_kernel");
 }
 
-int rlhf_gather_logprobs(const void* logits, long long stride_b, long long stride_t,
-                         const long long* ids, long long ids_stride_b, const int* lengths,
-                         int B, int T, int V, float* out_logprobs,
-                         void* workspace, size_t workspace_bytes, void* stream)
+int rlhf_gather_logprobs_ex(const void* logits, int logits_dtype, long long stride_b, long long stride_t,
+                            const long long* ids, long long ids_stride_b, const int* lengths,
+                            int B, int T, int V, float* out_logprobs, float* out_entropy,
+                            void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!logits || !ids || !lengths || !out_logprobs) return RLHF_ERR_NULL;
+    if (logits_dtype != RLHF_BF16 && logits_dtype != RLHF_F16) return RLHF_ERR_SCALAR;
     if (int e = check_shape(B, T, V)) return e;
     if (stride_b < 0 || stride_t < 0 || ids_stride_b < 0) return RLHF_ERR_STRIDE;
     if (T > 1 && stride_t < V) return RLHF_ERR_STRIDE;
-    if (!aligned(logits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) || !aligned(out_logprobs, 4))
+    if (!aligned(logits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) || !aligned(out_logprobs, 4) ||
+        (out_entropy && !aligned(out_entropy, 4)))
         return RLHF_ERR_ALIGN;
+    if (out_entropy && out_entropy == out_logprobs) return RLHF_ERR_STRIDE;
     if (int e = check_workspace(workspace, workspace_bytes, rlhf_workspace_bytes(B, T))) return e;
     DeviceInfo dev;
     if (int e = device_info(dev)) return e;
@@ -457,13 +482,24 @@ int rlhf_gather_logprobs(const void* logits, long long stride_b, long long strid
 
     WarpArgs wa{};
     wa.row = a;
+    wa.out_entropy = out_entropy;
+    const bool f16 = logits_dtype == RLHF_F16;
     if (rows_16B(logits, stride_b, stride_t, V)) {
-        if (int e = launch_warp_logprob<false, false>(wa, dev, (cudaStream_t)stream)) return e;
+        if (int e = launch_warp_logprob<false, false>(wa, f16, dev, (cudaStream_t)stream)) return e;
     } else {
         // rows that start or end off a 16-byte boundary (odd V, odd strides): same kernel, aligned spans
-        if (int e = launch_warp_logprob<false, true>(wa, dev, (cudaStream_t)stream)) return e;
+        if (int e = launch_warp_logprob<false, true>(wa, f16, dev, (cudaStream_t)stream)) return e;
     }
     return launch_check("logprob_warp_kernel");
+}
+
+int rlhf_gather_logprobs(const void* logits, long long stride_b, long long stride_t,
+                         const long long* ids, long long ids_stride_b, const int* lengths,
+                         int B, int T, int V, float* out_logprobs,
+                         void* workspace, size_t workspace_bytes, void* stream)
+{
+    return rlhf_gather_logprobs_ex(logits, RLHF_BF16, stride_b, stride_t, ids, ids_stride_b, lengths, B, T, V,
+                                   out_logprobs, nullptr, workspace, workspace_bytes, stream);
 }
 
 int rlhf_kl_reward(const float* lp_old, const float* lp_ref, const float* score, const int* lengths,
@@ -533,17 +569,45 @@ int rlhf_whiten_advantages(const float* adv, const int* lengths, int B, int T, f
     return launch_check("whiten_apply_kernel");
 }
 
-int rlhf_experience(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
-                    const void* ref_logits, long long ref_stride_b, long long ref_stride_t,
-                    const long long* ids, long long ids_stride_b, const int* lengths,
-                    const float* score, const float* values_old, const float* lp_old,
-                    int B, int T, int V, float beta_kl, float reward_clip, float gamma, float lambda,
-                    float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
-                    float* out_returns, void* workspace, size_t workspace_bytes, void* stream)
+int rlhf_ppo_stats(const float* lp_new, const float* lp_old, const float* adv, const int* lengths, int B, int T,
+                   float clip_eps, float* out_stats, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!lp_new || !lp_old || !adv || !lengths || !out_stats) return RLHF_ERR_NULL;
+    if (int e = check_shape(B, T, 1)) return e;
+    if (!(clip_eps > 0.f && clip_eps < 1.f)) return RLHF_ERR_SCALAR;
+    if (!aligned(lp_new, 4) || !aligned(lp_old, 4) || !aligned(adv, 4) || !aligned(lengths, 4) || !aligned(out_stats, 4))
+        return RLHF_ERR_ALIGN;
+    if (int e = check_workspace(workspace, workspace_bytes, rlhf_workspace_bytes(B, T))) return e;
+    char* ws = (char*)workspace;
+    StatsArgs a{};
+    a.lp_new = lp_new;
+    a.lp_old = lp_old;
+    a.adv = adv;
+    a.lengths = lengths;
+    a.B = B; a.T = T;
+    a.clip_eps = clip_eps;
+    a.out = out_stats;
+    a.ticket = (unsigned*)(ws + 4);
+    a.partials = (double*)(ws + kPartialsOffset);
+    const long long total = (long long)B * T;
+    const int grid = (int)std::min<long long>((total + 4095) / 4096, kWhitenMaxBlocks);
+    if (int e = keep_max_carveout(ppo_stats_kernel)) return e;
+    RLHF_CUDA(launch_kernel(ppo_stats_kernel, grid, kWhitenThreads, 0, (cudaStream_t)stream, a));
+    return launch_check("ppo_stats_kernel");
+}
+
+int rlhf_experience_ex(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
+                       const void* ref_logits, long long ref_stride_b, long long ref_stride_t, int logits_dtype,
+                       const long long* ids, long long ids_stride_b, const int* lengths,
+                       const float* score, const float* values_old, const float* lp_old,
+                       int B, int T, int V, float beta_kl, float reward_clip, float gamma, float lambda,
+                       float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
+                       float* out_returns, float* out_entropy, void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!actor_logits || !ref_logits || !ids || !lengths || !score || !values_old || !out_lp_actor ||
         !out_lp_ref || !out_rewards || !out_adv || !out_returns)
         return RLHF_ERR_NULL;
+    if (logits_dtype != RLHF_BF16 && logits_dtype != RLHF_F16) return RLHF_ERR_SCALAR;
     if (int e = check_shape(B, T, V)) return e;
     if (actor_stride_b < 0 || actor_stride_t < 0 || ref_stride_b < 0 || ref_stride_t < 0 || ids_stride_b < 0)
         return RLHF_ERR_STRIDE;
@@ -554,13 +618,14 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     if (!aligned(actor_logits, 2) || !aligned(ref_logits, 2) || !aligned(ids, 8) || !aligned(lengths, 4) ||
         !aligned(score, 4) || !aligned(values_old, 4) || (lp_old && !aligned(lp_old, 4)) ||
         !aligned(out_lp_actor, 4) || !aligned(out_lp_ref, 4) || !aligned(out_rewards, 4) ||
-        !aligned(out_adv, 4) || !aligned(out_returns, 4))
+        !aligned(out_adv, 4) || !aligned(out_returns, 4) || (out_entropy && !aligned(out_entropy, 4)))
         return RLHF_ERR_ALIGN;
     {
-        const float* outs[5] = {out_lp_actor, out_lp_ref, out_rewards, out_adv, out_returns};
-        for (int i = 0; i < 5; ++i) {
+        const float* outs[6] = {out_lp_actor, out_lp_ref, out_rewards, out_adv, out_returns, out_entropy};
+        for (int i = 0; i < 6; ++i) {
+            if (!outs[i]) continue;
             if (outs[i] == values_old || outs[i] == lp_old) return RLHF_ERR_STRIDE;
-            for (int j = i + 1; j < 5; ++j)
+            for (int j = i + 1; j < 6; ++j)
                 if (outs[i] == outs[j]) return RLHF_ERR_STRIDE;
         }
     }
@@ -585,11 +650,13 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     wa.stride2_b = ref_stride_b;
     wa.stride2_t = ref_stride_t;
     wa.out_lp2 = out_lp_ref;
+    wa.out_entropy = out_entropy;
+    const bool f16 = logits_dtype == RLHF_F16;
     cudaStream_t s = (cudaStream_t)stream;
     if (all_16B) {
-        if (int e = launch_warp_logprob<true, false>(wa, dev, s)) return e;
+        if (int e = launch_warp_logprob<true, false>(wa, f16, dev, s)) return e;
     } else {
-        if (int e = launch_warp_logprob<true, true>(wa, dev, s)) return e;
+        if (int e = launch_warp_logprob<true, true>(wa, f16, dev, s)) return e;
     }
     if (int e = launch_check("logprob_warp_kernel<dual>")) return e;
     if (int e = keep_max_carveout(reward_gae_kernel)) return e;
@@ -600,16 +667,32 @@ int rlhf_experience(const void* actor_logits, long long actor_stride_b, long lon
     return launch_check("reward_gae_kernel");
 }
 
-int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stride_t,
-                          const long long* ids, long long ids_stride_b, const int* lengths,
-                          const float* lp_old, const float* adv, const float* values_new,
-                          const float* values_old, const float* returns,
-                          int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
-                          float* out_loss_pg, float* out_loss_vf,
-                          void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
-                          float* out_dvalues, float* out_lp_new,
-                          void* workspace, size_t workspace_bytes, void* stream)
+int rlhf_experience(const void* actor_logits, long long actor_stride_b, long long actor_stride_t,
+                    const void* ref_logits, long long ref_stride_b, long long ref_stride_t,
+                    const long long* ids, long long ids_stride_b, const int* lengths,
+                    const float* score, const float* values_old, const float* lp_old,
+                    int B, int T, int V, float beta_kl, float reward_clip, float gamma, float lambda,
+                    float* out_lp_actor, float* out_lp_ref, float* out_rewards, float* out_adv,
+                    float* out_returns, void* workspace, size_t workspace_bytes, void* stream)
 {
+    return rlhf_experience_ex(actor_logits, actor_stride_b, actor_stride_t, ref_logits, ref_stride_b, ref_stride_t,
+                              RLHF_BF16, ids, ids_stride_b, lengths, score, values_old, lp_old, B, T, V, beta_kl,
+                              reward_clip, gamma, lambda, out_lp_actor, out_lp_ref, out_rewards, out_adv, out_returns,
+                              nullptr, workspace, workspace_bytes, stream);
+}
+
+int rlhf_ppo_loss_fwd_bwd_ex(const void* logits, int logits_dtype, long long stride_b, long long stride_t,
+                             const long long* ids, long long ids_stride_b, const int* lengths,
+                             const float* lp_old, const float* adv, const float* values_new,
+                             const float* values_old, const float* returns,
+                             int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
+                             float* out_loss_pg, float* out_loss_vf,
+                             void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                             float* out_dvalues, float* out_lp_new,
+                             void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (logits_dtype != RLHF_BF16 && logits_dtype != RLHF_F16) return RLHF_ERR_SCALAR;
+    const bool f16 = logits_dtype == RLHF_F16;
     if (int e = check_loss_args(logits, stride_b, stride_t, ids, ids_stride_b, lengths, lp_old, adv, values_new,
                                 values_old, returns, B, T, V, clip_eps, value_clip, grad_scale, out_loss_pg,
                                 out_loss_vf, out_dlogits, dl_stride_b, dl_stride_t, out_dvalues, out_lp_new))
@@ -647,7 +730,7 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
     const bool same_offsets = ((reinterpret_cast<uintptr_t>(out_dlogits) - reinterpret_cast<uintptr_t>(logits)) % 16) == 0 &&
                               ((dl_stride_b - stride_b) % 8) == 0 && ((dl_stride_t - stride_t) % 8) == 0;
     const bool ragged_fast = !all_16B && same_offsets && dbuf_applies(2u * (unsigned)V, dev, true);
-    if ((all_16B || ragged_fast) && dev.sm_count * 7 <= kMaxFusedBlocks) {
+    if (((all_16B && fast_loss_rows_apply(V, f16, dev)) || ragged_fast) && dev.sm_count * 7 <= kMaxFusedBlocks) {
         // fast path: the row kernel also does the finalisation (value loss, dvalues, loss reduction)
         a.fused = 1;
         a.values_new = values_new;
@@ -660,14 +743,15 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
         a.ticket = (unsigned*)(ws + 4);
         a.partials = (double*)(ws + kPartialsOffset);
         if (ragged_fast) {
-            if (int e = launch_dbuf<true>(a, dev, s)) return e;
+            if (int e = f16 ? launch_dbuf<true, true>(a, dev, s) : launch_dbuf<true, false>(a, dev, s)) return e;
         } else {
-            if (int e = launch_loss_rows(a, dev, s)) return e;
+            if (int e = launch_loss_rows(a, f16, dev, s)) return e;
         }
         return launch_check("loss row kernel");
     } else {
         int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * 8);
-        RLHF_CUDA(launch_kernel(row_generic_kernel<true>, grid, kGenericThreads, 0, s, a));
+        if (f16) RLHF_CUDA(launch_kernel(row_generic_kernel<true, true>, grid, kGenericThreads, 0, s, a));
+        else RLHF_CUDA(launch_kernel(row_generic_kernel<true, false>, grid, kGenericThreads, 0, s, a));
         if (int e = launch_check("row_generic_kernel<loss>")) return e;
     }
 
@@ -691,6 +775,22 @@ int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stri
     if (int e = keep_max_carveout(ppo_finalize_kernel)) return e;
     RLHF_CUDA(launch_kernel(ppo_finalize_kernel, fgrid, kFinalThreads, 0, s, f));
     return launch_check("ppo_finalize_kernel");
+}
+
+int rlhf_ppo_loss_fwd_bwd(const void* logits, long long stride_b, long long stride_t,
+                          const long long* ids, long long ids_stride_b, const int* lengths,
+                          const float* lp_old, const float* adv, const float* values_new,
+                          const float* values_old, const float* returns,
+                          int B, int T, int V, float clip_eps, float value_clip, float grad_scale,
+                          float* out_loss_pg, float* out_loss_vf,
+                          void* out_dlogits, long long dl_stride_b, long long dl_stride_t,
+                          float* out_dvalues, float* out_lp_new,
+                          void* workspace, size_t workspace_bytes, void* stream)
+{
+    return rlhf_ppo_loss_fwd_bwd_ex(logits, RLHF_BF16, stride_b, stride_t, ids, ids_stride_b, lengths, lp_old, adv,
+                                    values_new, values_old, returns, B, T, V, clip_eps, value_clip, grad_scale,
+                                    out_loss_pg, out_loss_vf, out_dlogits, dl_stride_b, dl_stride_t, out_dvalues,
+                                    out_lp_new, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -51,6 +51,36 @@ __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
 
 __device__ __forceinline__ float2 unpack_bf16x2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
 
+// The 16-bit element type of the logits and of their gradient: bf16 (kF16 = false) or IEEE binary16 (true).
+// Widening is exact; narrowing rounds to nearest even (and, for binary16, overflows to infinity above 65504).
+template <bool kF16>
+struct El {
+    static constexpr uint32_t kNegInf = kF16 ? 0xfc00u : 0xff80u;       // bit pattern of -inf
+    static constexpr uint32_t kNegInf2 = kNegInf | (kNegInf << 16);     // two of them
+    __device__ __forceinline__ static float widen(uint32_t bits16)
+    {
+        if (!kF16) return __uint_as_float(bits16 << 16);
+        float f;
+        asm("{\n\t.reg .b16 h;\n\tcvt.u16.u32 h, %1;\n\tcvt.f32.f16 %0, h;\n\t}" : "=f"(f) : "r"(bits16));
+        return f;
+    }
+    __device__ __forceinline__ static float2 unpack2(uint32_t w)
+    {
+        if (!kF16) return make_float2(bf16_lo(w), bf16_hi(w));
+        float2 r;
+        asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}"
+            : "=f"(r.x), "=f"(r.y) : "r"(w));
+        return r;
+    }
+    __device__ __forceinline__ static uint32_t pack2(float lo, float hi)
+    {
+        uint32_t r;
+        if (!kF16) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        else asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+};
+
 // Partial partition sum in the base-2 domain.
 struct Acc {
     float M;     // reference exponent

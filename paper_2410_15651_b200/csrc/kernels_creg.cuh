@@ -142,14 +142,15 @@ __device__ __noinline__ bool mbar_wait_cluster_slow(uint32_t bar, uint32_t parit
     }
 }
 
-// Entry j of a vector replaced by -inf (bf16 0xFF80).
+// Entry j of a vector replaced by -inf.
+template <bool kF16>
 __device__ __forceinline__ uint4 mask_vec_entry(const uint4& q, int j)
 {
     uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         if (i == j)
-            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | 0xff800000u) : ((w[i >> 1] & 0xffff0000u) | 0x0000ff80u);
+            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | (El<kF16>::kNegInf << 16)) : ((w[i >> 1] & 0xffff0000u) | El<kF16>::kNegInf);
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
@@ -189,8 +190,9 @@ __device__ __forceinline__ void tmem_wait_loads() { asm volatile("tcgen05.wait::
 
 // ---------------------------------------------------------------- the kernel
 // kTmem: a thread's vectors beyond the first kRegVecsTmem keep their exponentials in tensor memory; otherwise a
-// thread has at most kRegVecsOnly vectors and registers hold all of them.
-template <int NW, int kCluster, bool kTmem>
+// thread has at most kRegVecsOnly vectors and registers hold all of them.  kF16: logits and gradient are IEEE
+// binary16 instead of bf16.
+template <int NW, int kCluster, bool kTmem, bool kF16>
 __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
 {
     constexpr int kRegVecs = kTmem ? kRegVecsTmem : kRegVecsOnly;
@@ -243,7 +245,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
     // the vectors of every buffer past the end of the slice: -inf, a term of 0 in every sum
     for (int b = 0; b < NB; ++b)
         for (uint32_t v = nvec + tid; v < ca.buf_stride / 16u; v += kThreads)
-            ((uint4*)(smem + (size_t)b * ca.buf_stride))[v] = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            ((uint4*)(smem + (size_t)b * ca.buf_stride))[v] = make_uint4(El<kF16>::kNegInf2, El<kF16>::kNegInf2, El<kF16>::kNegInf2, El<kF16>::kNegInf2);
     fence_async_smem();
     if (kTmem) tmem_fence_before_sync();
     __syncthreads();
@@ -411,16 +413,16 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
         float Mref = kFloorM;
         if (nvec > 0) {
             uint4 q0 = *(const uint4*)rowbuf;
-            if (label_here && ylocal == 0) q0 = mask_vec_entry(q0, yj);
-            Mref = max8_scaled(q0);
+            if (label_here && ylocal == 0) q0 = mask_vec_entry<kF16>(q0, yj);
+            Mref = max8_scaled<kF16>(q0);
         }
         // The owner takes the generated token's logit out of the row (it becomes -inf, a term of 0), so that
         // the sums below are sums over the other entries and 1 - p_y comes without cancellation.
         float zy = 0.f, xy = kFloorM;
         if (owner) {
             uint16_t* slot = (uint16_t*)rowbuf + ((size_t)ylocal * 8 + yj);
-            zy = __uint_as_float((uint32_t)*slot << 16);
-            *slot = 0xff80u;
+            zy = El<kF16>::widen(*slot);
+            *slot = (uint16_t)El<kF16>::kNegInf;
             xy = fmaxf(zy * kLog2e, kFloorM);
         }
 
@@ -436,7 +438,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
                     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                     for (int h = 0; h < 4; ++h) {
-                        const float2 x = __ffma2_rn(unpack_bf16x2(w[h]), splat2(kLog2e), splat2(negM));
+                        const float2 x = __ffma2_rn(El<kF16>::unpack2(w[h]), splat2(kLog2e), splat2(negM));
                         e[j][h] = make_float2(ex2(x.x), ex2(x.y));
                     }
                     acc0 = __fadd2_rn(acc0, e[j][0]);
@@ -455,7 +457,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
                 float2 et[4];
 #pragma unroll
                 for (int h = 0; h < 4; ++h) {
-                    const float2 x = __ffma2_rn(unpack_bf16x2(w[h]), splat2(kLog2e), splat2(negM));
+                    const float2 x = __ffma2_rn(El<kF16>::unpack2(w[h]), splat2(kLog2e), splat2(negM));
                     et[h] = make_float2(ex2(x.x), ex2(x.y));
                 }
                 tmem_store8(tmem_addr + (uint32_t)j * 8u, et);
@@ -478,7 +480,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
             if (redo) {
                 // a reference of this thread's own: its largest scaled entry
                 float m = xy;
-                for (int j = 0; j < nj; ++j) m = fmaxf(m, max8_scaled(src[(size_t)j * kCons]));
+                for (int j = 0; j < nj; ++j) m = fmaxf(m, max8_scaled<kF16>(src[(size_t)j * kCons]));
                 M = m;
             }
         }
@@ -553,10 +555,10 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
 #pragma unroll
                 for (int h = 0; h < 4; ++h) {
                     const float2 d = __fmul2_rn(ev[h], sc2);
-                    o[h] = pack_bf16x2(d.x, d.y);
+                    o[h] = El<kF16>::pack2(d.x, d.y);
                 }
                 uint4 ov = make_uint4(o[0], o[1], o[2], o[3]);
-                if (j == jy) patch_label(ov, yj, dy);
+                if (j == jy) patch_label<kF16>(ov, yj, dy);
                 if (j < cnt) dst[(size_t)j * kCons] = ov;
             };
             if (kTmem) tmem_wait_stores();

@@ -89,7 +89,8 @@ __device__ __forceinline__ Acc dbuf_reduce(const Acc& a, float2* s_part, const L
 // even address and have any length.  The aligned span around the row is loaded; entries of its first and
 // last vector outside the row are skipped in pass 1 and never stored: the whole vectors inside the row go
 // out by bulk store, the ragged ends by 2-byte stores.
-template <int NW, bool kAny>
+// kF16: logits and gradient are IEEE binary16 instead of bf16.
+template <int NW, bool kAny, bool kF16 = false>
 __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
 {
     constexpr int kCons = NW * 32;
@@ -270,13 +271,13 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         // one vector of this thread, with whatever is special about it
         // (kAny) the first and last vector of the row, foreign entries turned into -inf; any other vector unchanged
         auto in_row = [&](const uint4& q, int j) {
-            if (kAny && j == jfirst) return mask_vec_outside(q, (int)eoff, 8);
-            if (kAny && j == jlast) return mask_vec_outside(q, 0, (int)((eoff + (uint32_t)p.V) & 7u));
+            if (kAny && j == jfirst) return mask_vec_outside<kF16>(q, (int)eoff, 8);
+            if (kAny && j == jlast) return mask_vec_outside<kF16>(q, 0, (int)((eoff + (uint32_t)p.V) & 7u));
             return q;
         };
         auto add_special = [&](Acc& acc, const uint4& q, int j, float& zy_out) {
-            if (j == jy) zy_out = acc_add_vec_label(acc, in_row(q, j), yj);
-            else acc_add_vec(acc, in_row(q, j));
+            if (j == jy) zy_out = acc_add_vec_label<kF16>(acc, in_row(q, j), yj);
+            else acc_add_vec<kF16>(acc, in_row(q, j));
         };
         const uint4* src = (const uint4*)(smem + (size_t)buf * da.row_stride) + tid;
 
@@ -286,7 +287,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
         // are summed without range handling and their sums checked afterwards, once per row: a thread that met
         // an entry 2^64 above the reference (or found no usable reference) redoes its share of the row with
         // the careful routines under a reference of its own, and the block then merges by the general rule.
-        const float Mref = max8_scaled(((const uint4*)(smem + (size_t)buf * da.row_stride))[(kAny && eoff != 0) ? 1 : 0]);
+        const float Mref = max8_scaled<kF16>(((const uint4*)(smem + (size_t)buf * da.row_stride))[(kAny && eoff != 0) ? 1 : 0]);
         Acc a = acc_empty();
         float zy = 0.f;
         bool redo = !(Mref > kFloorM);
@@ -304,11 +305,11 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
                 if ((unsigned)(jy - j) < 4u) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        if (j + u == jy) zy = acc_add_vec_label(a, q[u], yj);
-                        else acc_add_vec(a, q[u]);
+                        if (j + u == jy) zy = acc_add_vec_label<kF16>(a, q[u], yj);
+                        else acc_add_vec<kF16>(a, q[u]);
                     }
                 } else {
-                    const float vs = exp_sum_vecs<4>(q, -a.M);
+                    const float vs = exp_sum_vecs<4, kF16>(q, -a.M);
                     a.s += vs;
                     redo |= !(vs <= 1.8446744e19f);
                 }
@@ -364,18 +365,18 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_dbuf_kernel(DbufArgs da)
 #pragma unroll
                 for (int u = 0; u < 4; ++u) q[u] = src[(size_t)(j + u) * kCons];
                 uint4 o[4];
-                grad_vecs<4>(q, o, c2, sign2);
+                grad_vecs<4, kF16>(q, o, c2, sign2);
                 if ((unsigned)(jy - j) < 4u) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
-                        if (j + u == jy) patch_label(o[u], yj, dy);
+                        if (j + u == jy) patch_label<kF16>(o[u], yj, dy);
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) dst[(size_t)(j + u) * kCons] = o[u];
             }
             for (; j < cnt; ++j) {
-                uint4 o = grad_vec(src[(size_t)j * kCons], c2, sign2);
-                if (j == jy) patch_label(o, yj, dy);
+                uint4 o = grad_vec<kF16>(src[(size_t)j * kCons], c2, sign2);
+                if (j == jy) patch_label<kF16>(o, yj, dy);
                 dst[(size_t)j * kCons] = o;
             }
         }

@@ -55,7 +55,8 @@ __device__ inline Acc block_merge(Acc a, Acc* smem /* >= 32 */)
     return r;
 }
 
-template <bool kLoss>
+// kF16: logits and gradient are IEEE binary16 instead of bf16.
+template <bool kLoss, bool kF16 = false>
 __global__ void __launch_bounds__(kGenericThreads) row_generic_kernel(RowArgs p)
 {
     __shared__ Acc s_acc[32];
@@ -76,10 +77,10 @@ __global__ void __launch_bounds__(kGenericThreads) row_generic_kernel(RowArgs p)
         const uint16_t* row = p.logits + (long long)b * p.stride_b + (long long)t * p.stride_t;
 
         // every thread reads z_y before the block barrier, i.e. before any in-place write of this row
-        const float zy = __uint_as_float((uint32_t)row[y] << 16);
+        const float zy = El<kF16>::widen(row[y]);
         Acc a = acc_empty();
         for (int v = threadIdx.x; v < p.V; v += blockDim.x)
-            acc_add(a, __uint_as_float((uint32_t)row[v] << 16), v == (int)y);
+            acc_add(a, El<kF16>::widen(row[v]), v == (int)y);
         a = block_merge(a, s_acc);
         RowResult r = row_finish(a, zy);
 
@@ -101,10 +102,10 @@ __global__ void __launch_bounds__(kGenericThreads) row_generic_kernel(RowArgs p)
             const float c2 = log2f(fabsf(g)) - r.lse2;
             const uint16_t sign = g > 0.f ? 0x8000u : 0u;
             for (int v = threadIdx.x; v < p.V; v += blockDim.x) {
-                float z = __uint_as_float((uint32_t)row[v] << 16);    // read before the in-place write
+                float z = El<kF16>::widen(row[v]);                    // read before the in-place write
                 float d = ex2(fmaf(z, kLog2e, c2));
-                uint16_t h = (uint16_t)(pack_bf16x2(d, 0.f) & 0xffffu) ^ sign;
-                if (v == (int)y) h = (uint16_t)(pack_bf16x2(g * r.one_m_py, 0.f) & 0xffffu);
+                uint16_t h = (uint16_t)(El<kF16>::pack2(d, 0.f) & 0xffffu) ^ sign;
+                if (v == (int)y) h = (uint16_t)(El<kF16>::pack2(g * r.one_m_py, 0.f) & 0xffffu);
                 drow[v] = h;
             }
         }

@@ -126,21 +126,24 @@ __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(unsigned* sta
 }
 
 // ---------------------------------------------------------------- 8 logits at a time
+template <bool kF16 = false>
 __device__ __forceinline__ void unpack8(const uint4& q, float (&z)[8])
 {
-    z[0] = bf16_lo(q.x); z[1] = bf16_hi(q.x);
-    z[2] = bf16_lo(q.y); z[3] = bf16_hi(q.y);
-    z[4] = bf16_lo(q.z); z[5] = bf16_hi(q.z);
-    z[6] = bf16_lo(q.w); z[7] = bf16_hi(q.w);
+    const float2 a = El<kF16>::unpack2(q.x), b = El<kF16>::unpack2(q.y), c = El<kF16>::unpack2(q.z), d = El<kF16>::unpack2(q.w);
+    z[0] = a.x; z[1] = a.y;
+    z[2] = b.x; z[3] = b.y;
+    z[4] = c.x; z[5] = c.y;
+    z[6] = d.x; z[7] = d.y;
 }
 
 // Adds 8 entries none of which is the generated token.  The exponentials are formed against the
 // thread's current reference first; only if their sum is out of range (first vector of a thread, or
 // a logit more than 64 binades above the reference) is the reference raised and the vector redone.
+template <bool kF16 = false>
 __device__ __forceinline__ void acc_add_vec(Acc& a, const uint4& q)
 {
     float z[8], e[8];
-    unpack8(q, z);
+    unpack8<kF16>(q, z);
     float negM = -a.M;
 #pragma unroll
     for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(z[i], kLog2e, negM));
@@ -159,10 +162,11 @@ __device__ __forceinline__ void acc_add_vec(Acc& a, const uint4& q)
 }
 
 // The vector that holds the generated token (entry j): its term goes to a.ey; returns z_y.
+template <bool kF16 = false>
 __device__ __forceinline__ float acc_add_vec_label(Acc& a, const uint4& q, int j)
 {
     float z[8];
-    unpack8(q, z);
+    unpack8<kF16>(q, z);
     float zy = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -174,10 +178,11 @@ __device__ __forceinline__ float acc_add_vec_label(Acc& a, const uint4& q, int j
 
 // A vector of which only entries jlo <= j < jhi belong to the row (the first or last vector of a row that
 // does not start or end on a 16-byte boundary); entry jlabel, if in range, is the generated token.
+template <bool kF16 = false>
 __device__ __forceinline__ float acc_add_vec_range(Acc& a, const uint4& q, int jlo, int jhi, int jlabel)
 {
     float z[8];
-    unpack8(q, z);
+    unpack8<kF16>(q, z);
     float zy = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -189,43 +194,46 @@ __device__ __forceinline__ float acc_add_vec_range(Acc& a, const uint4& q, int j
     return zy;
 }
 
-// Entries of a vector outside [jlo, jhi) replaced by -inf (bf16 0xFF80): they then add nothing to a partition sum.
+// Entries of a vector outside [jlo, jhi) replaced by -inf: they then add nothing to a partition sum.
 // For the first or last vector of a row that does not start or end on a 16-byte boundary.
+template <bool kF16 = false>
 __device__ __forceinline__ uint4 mask_vec_outside(const uint4& q, int jlo, int jhi)
 {
     uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         if (i < jlo || i >= jhi)
-            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | 0xff800000u) : ((w[i >> 1] & 0xffff0000u) | 0x0000ff80u);
+            w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | (El<kF16>::kNegInf << 16)) : ((w[i >> 1] & 0xffff0000u) | El<kF16>::kNegInf);
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // dlogits for 8 entries: sign * 2^(x + c2), packed to bf16.  The scaling runs two entries at a time on
 // the packed fp32x2 FMA of sm_100; the exponentials stay on the special-function unit.
+template <bool kF16 = false>
 __device__ __forceinline__ uint4 grad_vec(const uint4& q, float c2, uint32_t sign2)
 {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
     uint32_t o[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        const float2 x = __ffma2_rn(unpack_bf16x2(w[k]), splat2(kLog2e), splat2(c2));
-        o[k] = pack_bf16x2(ex2(x.x), ex2(x.y)) ^ sign2;
+        const float2 x = __ffma2_rn(El<kF16>::unpack2(w[k]), splat2(kLog2e), splat2(c2));
+        o[k] = El<kF16>::pack2(ex2(x.x), ex2(x.y)) ^ sign2;
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-template <int U>
+template <int U, bool kF16 = false>
 __device__ __forceinline__ void grad_vecs(const uint4 (&q)[U], uint4 (&o)[U], float c2, uint32_t sign2)
 {
 #pragma unroll
-    for (int u = 0; u < U; ++u) o[u] = grad_vec(q[u], c2, sign2);
+    for (int u = 0; u < U; ++u) o[u] = grad_vec<kF16>(q[u], c2, sign2);
 }
 
+template <bool kF16 = false>
 __device__ __forceinline__ void patch_label(uint4& o, int j, float value)
 {
-    const uint32_t h = pack_bf16x2(value, 0.f) & 0xffffu;
+    const uint32_t h = El<kF16>::pack2(value, 0.f) & 0xffffu;
     const int ws = j >> 1;
     uint32_t w = ws == 0 ? o.x : (ws == 1 ? o.y : (ws == 2 ? o.z : o.w));
     w = (j & 1) ? ((w & 0x0000ffffu) | (h << 16)) : ((w & 0xffff0000u) | h);
@@ -311,7 +319,7 @@ __device__ __forceinline__ float sum_warp_sums(const float* s_sum)
 // ---------------------------------------------------------------- the kernel
 // Sum of the exponentials of U vectors against one reference exponent (no range check): scaling and
 // accumulation two entries at a time (packed fp32x2), one ex2 per entry.
-template <int U>
+template <int U, bool kF16 = false>
 __device__ __forceinline__ float exp_sum_vecs(const uint4 (&q)[U], float negM)
 {
     float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
@@ -320,17 +328,18 @@ __device__ __forceinline__ float exp_sum_vecs(const uint4 (&q)[U], float negM)
         const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const float2 x = __ffma2_rn(unpack_bf16x2(w[k]), splat2(kLog2e), splat2(negM));
+            const float2 x = __ffma2_rn(El<kF16>::unpack2(w[k]), splat2(kLog2e), splat2(negM));
             acc[k & 1] = __fadd2_rn(acc[k & 1], make_float2(ex2(x.x), ex2(x.y)));
         }
     }
     return (acc[0].x + acc[0].y) + (acc[1].x + acc[1].y);
 }
 
+template <bool kF16 = false>
 __device__ __forceinline__ float max8_scaled(const uint4& q)
 {
     float z[8];
-    unpack8(q, z);
+    unpack8<kF16>(q, z);
     float m = fmaxf(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])), fmaxf(fmaxf(z[4], z[5]), fmaxf(z[6], z[7])));
     return fmaxf(m * kLog2e, kFloorM);
 }

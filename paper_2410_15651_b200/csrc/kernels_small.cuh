@@ -231,6 +231,84 @@ __global__ void __launch_bounds__(256) whiten_apply_kernel(WhitenArgs p)
     }
 }
 
+// ---------------------------------------------------------------- monitors of the policy step
+// approx_kl = mean over valid tokens of (rho - 1) - log rho, clip_frac = share of valid tokens whose gradient the
+// clip switches off (clipped term strictly larger), rho = exp(lp_new - lp_old); from the O(B*T) arrays alone.
+// Same fixed-order reduction as the whitening statistics.
+struct StatsArgs {
+    const float* lp_new;
+    const float* lp_old;
+    const float* adv;
+    const int* lengths;
+    int B, T;
+    float clip_eps;
+    float* out;                 // device float[2]: approx_kl, clip_frac
+    unsigned* ticket;
+    double* partials;           // workspace: [kWhitenMaxBlocks][2]
+};
+
+__global__ void __launch_bounds__(kWhitenThreads) ppo_stats_kernel(StatsArgs p)
+{
+    __shared__ double s_red[2][kWhitenThreads / 32];
+    __shared__ long long s_n[kWhitenThreads / 32];
+    __shared__ bool s_last;
+    pdl_wait_prior_grid();
+    pdl_release_next_grid();
+    const long long total = (long long)p.B * p.T;
+    const long long per_block = (total + gridDim.x - 1) / gridDim.x;
+    const long long begin = per_block * blockIdx.x, end = min(total, begin + per_block);
+    double s1 = 0.0, s2 = 0.0;
+    for (long long i = begin + threadIdx.x; i < end; i += blockDim.x) {
+        const int b = (int)(i / p.T), t = (int)(i % p.T);
+        if (t < clamp_len(__ldg(p.lengths + b), p.T)) {
+            const float d = p.lp_new[i] - p.lp_old[i];
+            const float rho = expf(d);
+            s1 += (double)((rho - 1.f) - d);
+            const float A = p.adv[i];
+            const float unclipped = -A * rho;
+            const float clipped = -A * fminf(fmaxf(rho, 1.f - p.clip_eps), 1.f + p.clip_eps);
+            if (clipped > unclipped) s2 += 1.0;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_red[0][warp] = s1; s_red[1][warp] = s2; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, c = 0.0;
+        for (int w = 0; w < kWhitenThreads / 32; ++w) { a += s_red[0][w]; c += s_red[1][w]; }
+        p.partials[2 * blockIdx.x] = a;
+        p.partials[2 * blockIdx.x + 1] = c;
+        __threadfence();
+        s_last = (atomicAdd(p.ticket, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    long long n = 0;
+    for (int b = threadIdx.x; b < p.B; b += blockDim.x) n += clamp_len(__ldg(p.lengths + b), p.T);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+    if (lane == 0) s_n[warp] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        long long N = 0;
+        for (int w = 0; w < kWhitenThreads / 32; ++w) N += s_n[w];
+        double a = 0.0, c = 0.0;
+        for (unsigned k = 0; k < gridDim.x; ++k) {
+            a += ((volatile double*)p.partials)[2 * k];
+            c += ((volatile double*)p.partials)[2 * k + 1];
+        }
+        p.out[0] = N > 0 ? (float)(a / (double)N) : 0.f;
+        p.out[1] = N > 0 ? (float)(c / (double)N) : 0.f;
+        *p.ticket = 0u;
+    }
+}
+
 // ---------------------------------------------------------------- step 4: finalisation
 // Value loss and dvalues per token, then both losses summed in a fixed order: each block reduces a
 // contiguous range of tokens with a fixed tree, the last block to finish (a ticket in the workspace)

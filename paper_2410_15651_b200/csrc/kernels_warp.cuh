@@ -40,7 +40,74 @@ struct WarpArgs {
     const uint16_t* logits2;
     long long stride2_b, stride2_t;
     float* out_lp2;
+    // kEnt: entropy of the softmax of every valid row of the (first) tensor, 0 at padded positions
+    float* out_entropy;
 };
+
+// ---- sums that also carry what the entropy needs.  Beside (M, s, ey) of Acc a thread keeps
+//      ez = sum over the entries that are not the generated token of e * xr,   xr = max(x - M, -150),  e = 2^xr
+// (the clamp turns a deleted entry's -inf into a finite factor of a term that is 0 anyway).  Raising the reference
+// by d scales s and ey by 2^-d and turns ez into 2^-d * (ez - d * s).
+constexpr float kEntClamp = -150.f;
+
+__device__ __forceinline__ void acc_rebase_ent(Acc& a, float& ez, float newM)
+{
+    const float d = newM - a.M;
+    const float sc = ex2(-d);
+    ez = sc * (ez - d * a.s);
+    a.s *= sc;
+    a.ey *= sc;
+    a.M = newM;
+}
+
+__device__ __forceinline__ void acc_add_ent(Acc& a, float& ez, float z, bool is_label)
+{
+    const float x = z * kLog2e;
+    if (x - a.M > kRebase) acc_rebase_ent(a, ez, x);
+    const float xr = fmaxf(x - a.M, kEntClamp);
+    const float e = ex2(xr);
+    if (is_label) a.ey = e;
+    else { a.s += e; ez = fmaf(e, xr, ez); }
+}
+
+// Entries [jlo, jhi) of a vector, entry jlabel (if in range) being the generated token; returns its logit (else 0).
+template <bool kF16>
+__device__ __forceinline__ float acc_add_vec_ent(Acc& a, float& ez, const uint4& q, int jlo, int jhi, int jlabel)
+{
+    float z[8];
+    unpack8<kF16>(q, z);
+    float zy = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (i >= jlo && i < jhi) {
+            acc_add_ent(a, ez, z[i], i == jlabel);
+            if (i == jlabel) zy = z[i];
+        }
+    }
+    return zy;
+}
+
+// U whole vectors without the generated token against one reference: sum of e and sum of e * xr.
+template <int U, bool kF16>
+__device__ __forceinline__ float2 exp_sum_vecs_ent(const uint4 (&q)[U], float negM)
+{
+    float2 acc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    float2 accz[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float2 x = __ffma2_rn(El<kF16>::unpack2(w[k]), splat2(kLog2e), splat2(negM));
+            x.x = fmaxf(x.x, kEntClamp);
+            x.y = fmaxf(x.y, kEntClamp);
+            const float2 e = make_float2(ex2(x.x), ex2(x.y));
+            acc[k & 1] = __fadd2_rn(acc[k & 1], e);
+            accz[k & 1] = __ffma2_rn(e, x, accz[k & 1]);
+        }
+    }
+    return make_float2((acc[0].x + acc[0].y) + (acc[1].x + acc[1].y), (accz[0].x + accz[0].y) + (accz[1].x + accz[1].y));
+}
 
 inline size_t warp_kernel_smem_bytes(int warps_per_block)
 {
@@ -51,7 +118,8 @@ inline size_t warp_kernel_smem_bytes(int warps_per_block)
 // is then loaded as the 16-byte aligned span that contains it, and the entries of the first and last
 // vector that lie outside the row are skipped.  (The span stays inside the 16-byte blocks that hold the
 // row's first and last element.)
-template <int WPB, bool kDual, bool kAny>
+// kF16: the logits are IEEE binary16 instead of bf16.  kEnt: also write the entropy of every valid row.
+template <int WPB, bool kDual, bool kAny, bool kF16 = false, bool kEnt = false>
 __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -80,6 +148,7 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
             if (t >= clamp_len(__ldg(p.lengths + b), p.T)) {
                 p.out_lp[i] = 0.f;
                 if (kDual) wa.out_lp2[i] = 0.f;
+                if (kEnt) wa.out_entropy[i] = 0.f;
             }
         }
     }
@@ -175,23 +244,38 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
 
         Acc a = acc_empty();
         float zy = 0.f;
+        float ez = 0.f;                                             // kEnt only
         for (int c = 0; c < row_chunks; ++c) {
             mbar_wait(bar_addr + 8u * slot, (phases >> slot) & 1u, p.status, aborted, p.wait_limit_ns);
             phases ^= 1u << slot;
             const uint4* src = (const uint4*)(ring + (size_t)slot * kWarpChunk) + lane;
             if (c >= plain_begin && c < plain_end && c != ychunk) {
-                if (c == 0) a.M = max8_scaled(src[0]);             // this lane's reference exponent for the row
+                if (c == 0) {                                       // this lane's reference exponent for the row
+                    const float m0 = max8_scaled<kF16>(src[0]);
+                    if (kEnt) { if (m0 > kFloorM) a.M = m0; } else a.M = m0;
+                }
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint4 q[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) q[u] = src[(4 * h + u) * 32];
-                    const float vs = exp_sum_vecs<4>(q, -a.M);
-                    if (vs <= 1.8446744e19f) {
-                        a.s += vs;
-                    } else {
+                    if (kEnt) {
+                        const float2 vs = exp_sum_vecs_ent<4, kF16>(q, -a.M);
+                        if (vs.x <= 1.8446744e19f && a.M > kFloorM) {
+                            a.s += vs.x;
+                            ez += vs.y;
+                        } else {
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) acc_add_vec(a, q[u]);
+                            for (int u = 0; u < 4; ++u) acc_add_vec_ent<kF16>(a, ez, q[u], 0, 8, -1);
+                        }
+                    } else {
+                        const float vs = exp_sum_vecs<4, kF16>(q, -a.M);
+                        if (vs <= 1.8446744e19f) {
+                            a.s += vs;
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) acc_add_vec<kF16>(a, q[u]);
+                        }
                     }
                 }
             } else {
@@ -202,10 +286,12 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
                     if (v < row_vecs) {
                         const uint4 q = src[u * 32];
                         const int e0 = (int)(v * 8u) - (int)eoff;      // row index of the vector's first entry
-                        if (kAny && (e0 < 0 || e0 + 8 > p.V))
-                            zy += acc_add_vec_range(a, q, max(0, -e0), min(8, p.V - e0), v == yvec ? yj : -1);
-                        else if (v == yvec) zy = acc_add_vec_label(a, q, yj);
-                        else acc_add_vec(a, q);
+                        if (kEnt) {
+                            zy += acc_add_vec_ent<kF16>(a, ez, q, max(0, -e0), min(8, p.V - e0), v == yvec ? yj : -1);
+                        } else if (kAny && (e0 < 0 || e0 + 8 > p.V))
+                            zy += acc_add_vec_range<kF16>(a, q, max(0, -e0), min(8, p.V - e0), v == yvec ? yj : -1);
+                        else if (v == yvec) zy = acc_add_vec_label<kF16>(a, q, yj);
+                        else acc_add_vec<kF16>(a, q);
                     }
                 }
             }
@@ -225,10 +311,23 @@ __global__ void __launch_bounds__(WPB * 32, 1) logprob_warp_kernel(WarpArgs wa)
         const int owner = (int)(yvec & 31u);
         const float ey = __shfl_sync(0xffffffffu, a.ey * sc, owner);
         zy = __shfl_sync(0xffffffffu, zy, owner);
+        float ezw = 0.f;
+        if (kEnt) {
+            // every lane's ez against the common reference (see acc_rebase_ent), then the warp's sum
+            ezw = sc * (ez - (M - a.M) * a.s);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ezw += __shfl_xor_sync(0xffffffffu, ezw, o);
+        }
         if (lane == 0 && !aborted) {
             const RowResult r = row_finish(Acc{M, s, ey}, zy);
             float* out = (kDual && k >= N1) ? wa.out_lp2 : p.out_lp;
             out[flat] = bad_id ? 0.f : r.lp;
+            if (kEnt && !(kDual && k >= N1)) {
+                // H = ln2 * (log2 S - (sum_v e_v (x_v - M)) / S),  S = s + ey; the generated token's term joins the sum here
+                const float S = s + ey;
+                const float xyr = fmaxf(fmaf(zy, kLog2e, -M), kEntClamp);
+                wa.out_entropy[flat] = kLn2 * (log2f(S) - (ezw + ey * xyr) / S);
+            }
         }
     }
 }

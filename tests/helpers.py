@@ -5,7 +5,7 @@ Tolerances (fp32 arithmetic on the GPU against float64 on the CPU):
   log-probs                      |d| <= 1e-4
   rewards, advantages, returns,
   dvalues, losses                |d| <= 1e-4 * max(1, |x|)
-  dlogits (bf16)                 |d| <= ulp_bf16(x) + 1e-6
+  dlogits (bf16 / fp16)          |d| <= ulp(x) + 1e-6, ulp the spacing of the output type at x
 """
 from __future__ import annotations
 
@@ -19,8 +19,12 @@ TOL_REL = 1e-4
 
 
 def bits(x: torch.Tensor) -> np.ndarray:
-    """uint16 bit patterns of a bf16 tensor (copied to the CPU if needed), strides preserved."""
-    return inputs.bf16_bits(x.cpu() if x.is_cuda else x)
+    """What the oracle takes for a 16-bit logits tensor (copied to the CPU if needed, strides preserved): uint16 bit
+    patterns for bf16, a numpy float16 array for fp16."""
+    x = x.cpu() if x.is_cuda else x
+    if x.dtype == torch.float16:
+        return x.numpy()
+    return inputs.bf16_bits(x)
 
 
 def np32(x: torch.Tensor) -> np.ndarray:
@@ -111,7 +115,7 @@ def check_dlogits_rows(oracle, run: OracleRun, logits: torch.Tensor, ids: torch.
         want = oracle.dlogits_rows(bits(z), np.ascontiguousarray(sub_ids), sub_len, sub_g,
                                    np.arange(rr.size))
         got = dlogits[bsel, tsel].float().cpu().numpy().astype(np.float64)
-        lim = oracle.bf16_ulp(want) + 1e-6
+        lim = (oracle.f16_ulp(want) if dlogits.dtype == torch.float16 else oracle.bf16_ulp(want)) + 1e-6
         err = np.abs(got - want)
         assert np.isfinite(got).all()
         ratio = float((err / lim).max(initial=0.0))

@@ -114,7 +114,11 @@ def dlogits_properties(run, out, ids, logits):
         if pad.any():
             assert (d[b][pad].view(torch.int16) == 0).all()         # exact +0
         rs = db.double().sum(-1).abs()
-        lim = 0.5 * db.abs().double().sum(-1) * 2.0 ** -7 + 1e-5    # sum of half-ulps bound, with slack
+        if d.dtype == torch.float16:
+            # half a step of every entry: relative 2^-11 for normal values, 2^-25 absolute below 2^-14
+            lim = 0.5 * db.abs().double().sum(-1) * 2.0 ** -10 + V * 2.0 ** -25 + 1e-5
+        else:
+            lim = 0.5 * db.abs().double().sum(-1) * 2.0 ** -7 + 1e-5    # sum of half-ulps bound, with slack
         assert (rs <= lim).all(), (b, float((rs / lim).max()))
         g = torch.as_tensor(run.ppo.g[b], device=d.device)
         dy = db.gather(1, ids[b][:, None])[:, 0].double()
