@@ -306,7 +306,8 @@ int rlhf_ppo_stats(const float* lp_new, const float* lp_old, const float* adv, c
  *    A larger batch is refused with RLHF_ERR_TOO_LARGE and nothing is launched.
  *  - The call allocates and frees nothing, directly or through any library.
  *  - The first call on each device looks up the device address of the array (with that device
- *    current) and remembers it.  Make that first call outside any stream capture.
+ *    current) and remembers it.  Make that first call outside any stream capture.  The remembered
+ *    address does not survive a cudaDeviceReset in the same process.
  *  - All calls on one device share the array, and it keeps what the previous call left in it.
  *    The call itself clears the words that must start at zero.  Two calls whose kernels can run
  *    at the same time on one device (different streams without an ordering between them) race on
