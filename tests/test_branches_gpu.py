@@ -232,3 +232,48 @@ def test_sequence_shards_reproduce_the_whole_batch(oracle, name, kw, shards):
     total = acc / n_global
     assert close_rel(total[0].item(), run.ppo.loss_pg)[0] and close_rel(total[1].item(), run.ppo.loss_vf)[0]
     assert close_rel(total[0].item(), float(whole.loss[0]))[0]
+
+
+@pytest.mark.parametrize("V", [8192, 8200, 16384, 32768, 32776, 45056, 53248, 57344, 98304, 114688, 163840])
+def test_vocabulary_sizes_around_the_kernel_boundaries(oracle, V):
+    # 16 KB rows (the first size of the on-chip-exponentials kernel), rows that fill a thread's register-held vectors
+    # exactly and by one more vector (tensor memory), the last size one block holds twice and the first that needs a
+    # cluster of 2, 3, 4 blocks
+    from test_parity_gpu import run_steps
+    w = inputs.scaled(inputs.WORKLOADS["ragged"], V=V, B=3, T=5, seed=200 + V % 13)
+    batch = inputs.make_batch(w, device=DEV)
+    batch["lengths"] = torch.tensor([5, 0, 3], dtype=torch.int32, device=DEV)
+    batch["ids"][0, 0], batch["ids"][0, 1] = 0, V - 1               # labels in the first and the last vector
+    batch["actor"][0, 0, 0], batch["actor"][0, 1, V - 1] = 2.0, 3.0
+    batch["ref"][0, :2] = batch["actor"][0, :2]
+    run = OracleRun(oracle, w, batch)
+    run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"], all_rows=True)
+
+
+@pytest.mark.parametrize("V", [32000, 50272, 128256])
+def test_all_padding_and_prompt_views_on_the_main_loss_kernel(oracle, V):
+    from test_parity_gpu import run_steps
+    # no valid token at all: every row is zero-filled, both losses are 0
+    w0 = inputs.scaled(inputs.WORKLOADS["llama2"], V=V, B=2, T=4, P=3, lengths="uniform:0:0")
+    b0 = inputs.make_batch(w0, device=DEV)
+    run0 = OracleRun(oracle, w0, b0)
+    out, _ = run_steps(oracle, w0, b0, run0, b0["actor"], b0["ref"], b0["ids"], all_rows=True)
+    assert (out.loss == 0).all() and (out.dlogits.view(torch.int16) == 0).all() and (out.dvalues == 0).all()
+    # the response rows as a strided view of a [B,P+T,V] tensor, out of place and in place on the view itself
+    w = inputs.scaled(inputs.WORKLOADS["llama2"], V=V, B=2, T=4, P=3, lengths="uniform:2:4")
+    full = inputs.make_batch(w, device=DEV, with_prompt=True)
+    logits, ref, ids = inputs.response_view(w, full["actor"]), inputs.response_view(w, full["ref"]), full["ids"][:, w.P:]
+    assert not logits.is_contiguous()
+    run = OracleRun(oracle, w, full, logits_view=logits, ref_view=ref, ids_view=ids)
+    run_steps(oracle, w, full, run, logits, ref, ids, all_rows=True)
+    full2 = full["actor"].clone()
+    view2 = inputs.response_view(w, full2)
+    ws = binding.workspace(w.B, w.T, DEV)
+    out2 = binding.PPOOutputs(view2, in_place=True)
+    lp_old, adv, vn, vo, ret = _loss_inputs(run)
+    binding.ppo_loss_fwd_bwd(view2, ids, full["lengths"], lp_old, adv, vn, vo, ret, w.clip_eps, w.value_clip,
+                             run.grad_scale, ws, out2)
+    assert binding.poll_status(ws) == 0
+    assert torch.equal(full2[:, :w.P - 1], full["actor"][:, :w.P - 1])            # the prompt rows around it are untouched
+    assert torch.equal(full2[:, w.P - 1 + w.T:], full["actor"][:, w.P - 1 + w.T:])
+    check_dlogits_rows(oracle, run, logits, ids, view2, np.arange(w.B * w.T))
