@@ -12,7 +12,6 @@
 #include "common.cuh"
 #include "kernels_generic.cuh"
 #include "kernels_ring.cuh"
-#include "kernels_dbuf.cuh"
 #include "kernels_creg.cuh"
 #include "kernels_warp.cuh"
 #include "kernels_small.cuh"
@@ -167,29 +166,6 @@ int launch_warp_logprob(const WarpArgs& wa, bool f16, const DeviceInfo& dev, cud
                : launch_warp_logprob_as<kDual, kAny, false, false>(wa, dev, s);
 }
 
-constexpr int kDbufWarps = 16;
-
-// Loss kernel for rows of which two fit in shared memory; returns false if the row is out of its range.
-bool dbuf_applies(unsigned row_bytes, const DeviceInfo& dev, bool any_alignment = false)
-{
-    return row_bytes >= 16384 && dbuf_smem_bytes(row_bytes, any_alignment) + 1280 <= (size_t)dev.max_smem_optin;
-}
-
-template <bool kAny, bool kF16>
-int launch_dbuf(const RowArgs& a, const DeviceInfo& dev, cudaStream_t s)
-{
-    DbufArgs da{};
-    da.row = a;
-    da.row_bytes = 2u * (unsigned)a.V;
-    da.row_stride = (unsigned)dbuf_row_stride(da.row_bytes, kAny);
-    const size_t smem = dbuf_smem_bytes(da.row_bytes, kAny);
-    const long long rows = (long long)a.B * a.T;
-    const int grid = (int)std::min<long long>(rows, dev.sm_count);
-    RLHF_CUDA(cudaFuncSetAttribute(loss_dbuf_kernel<kDbufWarps, kAny, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    RLHF_CUDA(launch_kernel(loss_dbuf_kernel<kDbufWarps, kAny, kF16>, grid, kDbufWarps * 32 + 32, smem, s, da));
-    return RLHF_OK;
-}
-
 // Loss kernel that keeps a row's exponentials on chip (kernels_creg.cuh): in registers if a consumer thread has at
 // most kRegVecsOnly vectors of a row, else in registers for its first kRegVecsTmem vectors and in tensor memory for
 // up to kTmemVecs more.  A block holds two buffers of its share of
@@ -231,7 +207,7 @@ CregPlan plan_creg(unsigned row_bytes, const DeviceInfo& dev)
 
 // Clusters of the kernel that the device holds at once (one block per SM); looked up once per device and
 // cluster size.  It only sizes the persistent grid: a larger grid would still be correct.
-template <int NW, int C, bool kTmem, bool kF16>
+template <int NW, int C, bool kTmem, bool kF16, bool kAny>
 int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
 {
     if (C == 1) { out = dev.sm_count; return RLHF_OK; }
@@ -245,7 +221,7 @@ int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attr[2];
         fill_launch_config(cfg, attr, dev.sm_count / C * C, NW * 32 + 32, pl.smem_bytes, C, nullptr);
-        RLHF_CUDA(cudaOccupancyMaxActiveClusters(&n, loss_creg_kernel<NW, C, kTmem, kF16>, &cfg));
+        RLHF_CUDA(cudaOccupancyMaxActiveClusters(&n, loss_creg_kernel<NW, C, kTmem, kF16, kAny>, &cfg));
         if (n < 1) n = 1;
         if (d < 0 || d >= 64) { out = n; return RLHF_OK; }
         cached[d] = n;
@@ -254,7 +230,7 @@ int creg_resident_clusters(const CregPlan& pl, const DeviceInfo& dev, int& out)
     return RLHF_OK;
 }
 
-template <int NW, int C, bool kTmem, bool kF16>
+template <int NW, int C, bool kTmem, bool kF16, bool kAny = false>
 int launch_creg(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cudaStream_t s)
 {
     CregArgs ca{};
@@ -265,13 +241,13 @@ int launch_creg(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cud
     ca.tmem_cols = pl.tmem_cols;
     ca.n_buf = pl.n_buf;
     ca.row_counter = (unsigned*)((char*)a.status + 16);
-    RLHF_CUDA(cudaFuncSetAttribute(loss_creg_kernel<NW, C, kTmem, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    RLHF_CUDA(cudaFuncSetAttribute(loss_creg_kernel<NW, C, kTmem, kF16, kAny>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)pl.smem_bytes));
     int clusters = 0;
-    if (int e = creg_resident_clusters<NW, C, kTmem, kF16>(pl, dev, clusters)) return e;
+    if (int e = creg_resident_clusters<NW, C, kTmem, kF16, kAny>(pl, dev, clusters)) return e;
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, clusters) * C;
-    RLHF_CUDA(launch_kernel_cluster(loss_creg_kernel<NW, C, kTmem, kF16>, grid, NW * 32 + 32, pl.smem_bytes, C, s, ca));
+    RLHF_CUDA(launch_kernel_cluster(loss_creg_kernel<NW, C, kTmem, kF16, kAny>, grid, NW * 32 + 32, pl.smem_bytes, C, s, ca));
     return RLHF_OK;
 }
 
@@ -286,8 +262,25 @@ int launch_creg_cluster(const RowArgs& a, const CregPlan& pl, const DeviceInfo& 
     }
 }
 
-// The loss row kernel for 16-byte aligned rows: exponentials in registers where the row (or its share in a
-// cluster) fits, else two resident rows, else the chunk ring.
+// The loss row kernel for 16-byte aligned rows: exponentials kept on chip where the row (or its share in a
+// cluster) fits, else the chunk ring.
+// Rows off 16-byte boundaries: the kernel loads the aligned span around a row, at most 14 bytes before it and 14 after;
+// only single blocks take such rows.
+CregPlan plan_creg_any(int V, const DeviceInfo& dev)
+{
+    const unsigned span = (14u + 2u * (unsigned)V + 15u) & ~15u;
+    CregPlan pl = plan_creg(span, dev);
+    if (pl.cluster != 1) pl.cluster = 0;
+    return pl;
+}
+
+template <bool kF16>
+int launch_creg_any(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev, cudaStream_t s)
+{
+    return pl.tmem_cols != 0 ? launch_creg<kCregWarps, 1, true, kF16, true>(a, pl, dev, s)
+                             : launch_creg<kCregWarps, 1, false, kF16, true>(a, pl, dev, s);
+}
+
 // The fast loss kernels for 16-byte aligned rows of this length (binary16 rows: the on-chip-exponentials kernel
 // only; the chunk ring is a bf16 kernel).
 bool fast_loss_rows_apply(int V, bool f16, const DeviceInfo& dev)
@@ -306,7 +299,6 @@ int launch_loss_rows(const RowArgs& a, bool f16, const DeviceInfo& dev, cudaStre
         return cp.tmem_cols != 0 ? launch_creg_cluster<kCregWarps, true, false>(a, cp, dev, s)
                                  : launch_creg_cluster<kCregWarps, false, false>(a, cp, dev, s);
     }
-    if (dbuf_applies(row_bytes, dev)) return launch_dbuf<false, false>(a, dev, s);
     const RingPlan pl = plan_ring(row_bytes, dev.smem_per_sm, dev.max_smem_optin);
     RingArgs ra{};
     ra.row = a;
@@ -725,11 +717,12 @@ int rlhf_ppo_loss_fwd_bwd_ex(const void* logits, int logits_dtype, long long str
     cudaStream_t s = (cudaStream_t)stream;
     long long rows = (long long)B * T;
     const bool all_16B = rows_16B(logits, stride_b, stride_t, V) && rows_16B(out_dlogits, dl_stride_b, dl_stride_t, V);
-    // rows off 16-byte boundaries can still take the two-resident-rows kernel if every dlogits row is as far
-    // off a boundary as its logits row (in place, or a second tensor of the same layout)
+    // rows off 16-byte boundaries can still take the fast kernel if every dlogits row is as far off a boundary as
+    // its logits row (in place, or a second tensor of the same layout)
     const bool same_offsets = ((reinterpret_cast<uintptr_t>(out_dlogits) - reinterpret_cast<uintptr_t>(logits)) % 16) == 0 &&
                               ((dl_stride_b - stride_b) % 8) == 0 && ((dl_stride_t - stride_t) % 8) == 0;
-    const bool ragged_fast = !all_16B && same_offsets && dbuf_applies(2u * (unsigned)V, dev, true);
+    const CregPlan any_plan = plan_creg_any(V, dev);
+    const bool ragged_fast = !all_16B && same_offsets && any_plan.cluster == 1;
     if (((all_16B && fast_loss_rows_apply(V, f16, dev)) || ragged_fast) && dev.sm_count * 7 <= kMaxFusedBlocks) {
         // fast path: the row kernel also does the finalisation (value loss, dvalues, loss reduction)
         a.fused = 1;
@@ -743,7 +736,7 @@ int rlhf_ppo_loss_fwd_bwd_ex(const void* logits, int logits_dtype, long long str
         a.ticket = (unsigned*)(ws + 4);
         a.partials = (double*)(ws + kPartialsOffset);
         if (ragged_fast) {
-            if (int e = f16 ? launch_dbuf<true, true>(a, dev, s) : launch_dbuf<true, false>(a, dev, s)) return e;
+            if (int e = f16 ? launch_creg_any<true>(a, any_plan, dev, s) : launch_creg_any<false>(a, any_plan, dev, s)) return e;
         } else {
             if (int e = launch_loss_rows(a, f16, dev, s)) return e;
         }

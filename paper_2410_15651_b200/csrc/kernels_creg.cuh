@@ -3,17 +3,19 @@
 // cluster of up to 4 blocks.
 //
 // A row's gradient needs every softmax term twice: once in the partition sum and once, scaled by the
-// token's g / sum, as the gradient entry itself.  The two-resident-rows kernel recomputes the
-// exponential in the second pass: two ex2 per logit, which makes the special-function unit (16 results
-// per clock per SM) the limiter whenever the SM clock drops under the power cap.  Here every consumer
+// token's g / sum, as the gradient entry itself.  Recomputing the exponential in the second pass costs two
+// ex2 per logit, which makes the special-function unit (16 results per clock per SM) the limiter
+// whenever the SM clock drops under the power cap.  Here every consumer
 // thread keeps the exponentials of its share of the row after the first pass -- those of its first
 // kRegVecs vectors in registers, those of the following ones in tensor memory (the 256 KB per SM that
 // otherwise hold tensor-core accumulators; each warp stores and loads its own 32 lanes x 128 columns with
 // tcgen05.st / tcgen05.ld) -- so the second pass is one packed multiply and one conversion per pair of
 // logits: one ex2 per logit in total, and no second read of the row from shared memory.
 //
-// Rows up to about 110 KB are held by one block (two row buffers, as in the two-resident-rows kernel; three
-// where they fit, which keeps more loads in flight).
+// Rows up to about 105 KB are held by one block, in two row buffers (three where they fit, which keeps more
+// loads in flight): while row i is reduced (pass 1) and turned into dlogits (pass 2) out of one buffer, the
+// bulk copies of the next rows into the others are already in flight, so that DRAM sees each row read once
+// and written once and, but for a block's first row, the consumers find their row in shared memory.
 // Longer rows are cut into kCluster contiguous slices, one per block of a cluster: every block runs the
 // pipeline on its slice (its own producer thread, its own two slice buffers), and once per row the blocks
 // exchange their partial partition sums through distributed shared memory (one asynchronous 16-byte store
@@ -37,9 +39,55 @@
 // block drain.  The tensor-memory columns are released by the warp that took them, after all consumers
 // have passed a block barrier at the end of the kernel.
 #pragma once
-#include "kernels_dbuf.cuh"
+#include "kernels_ring.cuh"
 
 namespace rlhf {
+
+constexpr long long kTailPads = 2;      // padded rows of a cluster that are zero-filled after its last load
+
+// What the producer publishes for each row before it arms the row's "landed" barrier.
+struct RowInfo {
+    long long flat;         // b*T + t
+    long long dl_offset;    // element offset of the dlogits row
+    int y;                  // generated token (0 if it was out of range)
+    int bad_id;
+    float lp_old;
+    float adv;
+    unsigned mis;           // bytes between the 16-byte boundary below the row's first logit and that logit
+    unsigned pad;
+};
+
+// Block-wide total of the partial sums, as consumer_reduce but with log2(NW) cross-warp steps.
+template <int NW>
+__device__ __forceinline__ Acc creg_reduce(const Acc& a, float2* s_part, const LabelInfo* s_lab, int warp, int lane)
+{
+    float M = a.M;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float s = a.s * ex2(a.M - M);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) s_part[warp] = make_float2(M, s);
+    asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+    constexpr int kTop = NW > 16 ? 16 : (NW > 8 ? 8 : 4);
+    const float2 pw = lane < NW ? s_part[lane] : make_float2(kFloorM, 0.f);
+    float Mt = pw.x;
+#pragma unroll
+    for (int o = kTop; o > 0; o >>= 1) Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, o));
+    float st = pw.y * ex2(pw.x - Mt);
+#pragma unroll
+    for (int o = kTop; o > 0; o >>= 1) st += __shfl_xor_sync(0xffffffffu, st, o);
+    // lanes >= 2*kTop did not take part; everyone takes lane 0's result
+    Mt = __shfl_sync(0xffffffffu, Mt, 0);
+    st = __shfl_sync(0xffffffffu, st, 0);
+    const LabelInfo li = *s_lab;
+    Acc tot;
+    tot.M = fmaxf(Mt, li.M);
+    tot.s = st * ex2(Mt - tot.M);
+    tot.ey = li.ey * ex2(li.M - tot.M);
+    return tot;
+}
+
 
 #ifndef RLHF_CREG_REGVECS_ONLY
 #define RLHF_CREG_REGVECS_ONLY 8
@@ -191,10 +239,15 @@ __device__ __forceinline__ void tmem_wait_loads() { asm volatile("tcgen05.wait::
 // ---------------------------------------------------------------- the kernel
 // kTmem: a thread's vectors beyond the first kRegVecsTmem keep their exponentials in tensor memory; otherwise a
 // thread has at most kRegVecsOnly vectors and registers hold all of them.  kF16: logits and gradient are IEEE
-// binary16 instead of bf16.
-template <int NW, int kCluster, bool kTmem, bool kF16>
+// binary16 instead of bf16.  kAny (single blocks only): rows, of logits and dlogits alike and with the same offset
+// from a 16-byte boundary, may start at any even address and have any length; the aligned span around a row is
+// loaded, the entries of its first and last vector that belong to neighbouring rows are turned into -inf in the
+// buffer before the first pass, and only the row's own bytes are stored: whole vectors by bulk store, the ragged
+// ends by 2-byte stores.
+template <int NW, int kCluster, bool kTmem, bool kF16, bool kAny = false>
 __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
 {
+    static_assert(!kAny || kCluster == 1, "rows off 16-byte boundaries are not split over a cluster");
     constexpr int kRegVecs = kTmem ? kRegVecsTmem : kRegVecsOnly;
     constexpr int kCons = NW * 32;
     constexpr int kThreads = kCons + 32;
@@ -219,7 +272,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
     const uint32_t crank = kCluster > 1 ? cluster_ctarank() : 0u;
     const long long cid = blockIdx.x / kCluster;             // this block's cluster
     const long long G = gridDim.x / kCluster;                // clusters in the grid
-    const uint32_t row_vecs = ca.row_bytes / 16u;
+    const uint32_t row_vecs = kAny ? ca.slice_vecs : ca.row_bytes / 16u;   // kAny: the longest aligned span around a row
     const uint32_t v0 = min(row_vecs, crank * ca.slice_vecs);      // this block's slice of every row: vectors [v0, v0+nvec)
     const uint32_t nvec = min(row_vecs - v0, ca.slice_vecs);
     const uint32_t slice_off = v0 * 16u, slice_bytes = nvec * 16u;
@@ -271,8 +324,16 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
             long long pads_done = 0;
             auto zero_fill_row = [&](int b, int t) {
                 unsigned char* drow = (unsigned char*)(p.dlogits + (long long)b * p.dl_stride_b + (long long)t * p.dl_stride_t) + slice_off;
-                for (uint32_t off = 0; off < slice_bytes; off += kCregZeroBytes)
-                    bulk_store(drow + off, smem_u32(zero_buf), min((uint32_t)kCregZeroBytes, slice_bytes - off));
+                uint32_t lo = 0, hi = slice_bytes;                   // [lo,hi): the part of the row made of whole 16-byte vectors
+                if (kAny) {
+                    const uint32_t mis = (uint32_t)((uintptr_t)drow & 15u);
+                    lo = min(ca.row_bytes, (16u - mis) & 15u);
+                    hi = max(lo, ca.row_bytes - ((mis + ca.row_bytes) & 15u));
+                    for (uint32_t o = 0; o < lo; o += 2) *(uint16_t*)(drow + o) = 0;
+                    for (uint32_t o = hi; o < ca.row_bytes; o += 2) *(uint16_t*)(drow + o) = 0;
+                }
+                for (uint32_t off = lo; off < hi; off += kCregZeroBytes)
+                    bulk_store(drow + off, smem_u32(zero_buf), min((uint32_t)kCregZeroBytes, hi - off));
                 bulk_commit();
             };
             auto zero_fill_next = [&]() {
@@ -288,8 +349,19 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
                 if (aborted) return;
                 const uint32_t srcb = buf_addr + (uint32_t)buf * ca.buf_stride;
                 unsigned char* drow = (unsigned char*)(p.dlogits + s_row[buf].dl_offset) + slice_off;
-                for (uint32_t off = 0; off < slice_bytes; off += kPiece)
-                    bulk_store(drow + off, srcb + off, min(kPiece, slice_bytes - off));
+                uint32_t mis = 0, lo = 0, hi = slice_bytes;          // row = span bytes [mis, mis + row_bytes); whole vectors [lo,hi)
+                if (kAny) {
+                    mis = (uint32_t)((uintptr_t)drow & 15u);
+                    lo = (mis + 15u) & ~15u;
+                    hi = (mis + ca.row_bytes) & ~15u;
+                    if (hi < lo) hi = lo;
+                    const unsigned char* sb = smem + (size_t)buf * ca.buf_stride;
+                    for (uint32_t o = mis; o < min(lo, mis + ca.row_bytes); o += 2) *(uint16_t*)(drow - mis + o) = *(const uint16_t*)(sb + o);
+                    for (uint32_t o = max(hi, mis); o < mis + ca.row_bytes; o += 2) *(uint16_t*)(drow - mis + o) = *(const uint16_t*)(sb + o);
+                    fence_async_smem();                              // these reads, before the buffer is refilled by bulk copies
+                }
+                for (uint32_t off = lo; off < hi; off += kPiece)
+                    bulk_store(drow - mis + off, srcb + off, min(kPiece, hi - off));
                 bulk_commit();
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             };
@@ -343,7 +415,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
                 ri.y = ri.bad_id ? 0 : (int)a.y;
                 ri.lp_old = a.lp_old;
                 ri.adv = a.adv;
-                ri.mis = 0;
+                ri.mis = kAny ? (unsigned)((uintptr_t)row & 15u) : 0u;
                 ri.pad = 0;
                 if (ri.bad_id && crank == 0) atomicOr(p.status, kErrIdRange);
                 const int buf = i % NB;
@@ -351,9 +423,11 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
                 if (aborted) break;
                 s_row[buf] = ri;
                 const uint32_t dst = buf_addr + (uint32_t)buf * ca.buf_stride;
-                mbar_arrive_expect_tx(landed(buf), slice_bytes);         // release: publishes s_row[buf]
-                for (uint32_t off = 0; off < slice_bytes; off += kPiece)
-                    bulk_load(dst + off, row + off, min(kPiece, slice_bytes - off), landed(buf));
+                // kAny: the aligned span around the row (it stays inside the 16-byte blocks that hold the row's ends)
+                const uint32_t load_bytes = kAny ? ((ri.mis + ca.row_bytes + 15u) & ~15u) : slice_bytes;
+                mbar_arrive_expect_tx(landed(buf), load_bytes);          // release: publishes s_row[buf]
+                for (uint32_t off = 0; off < load_bytes; off += kPiece)
+                    bulk_load(dst + off, row - ri.mis + off, min(kPiece, load_bytes - off), landed(buf));
                 if (kCluster > 1) {
                     const long long target = ((long long)(i + 1) * pads_early) / n_mine;
                     while (pads_done < target) { zero_fill_next(); ++pads_done; }
@@ -401,9 +475,21 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
         unsigned char* rowbuf = smem + (size_t)buf * ca.buf_stride;
         const uint4* src = (const uint4*)rowbuf + tid;
 
+        // kAny: eoff entries of the buffer's first vector precede the row; they, the entries after the row's end in its
+        // last vector and the vector after that (left from a longer span) are not the row's: their owners make them -inf
+        const uint32_t eoff = kAny ? (ri.mis >> 1) : 0u;
+        if (kAny) {
+            const uint32_t end = eoff + (uint32_t)p.V;               // entry index, in the buffer, of the row's end
+            const uint32_t last = (end - 1) >> 3, past = last + 1;   // vector of the last entry, and the one after it
+            uint4* vecs = (uint4*)rowbuf;
+            if (eoff != 0 && tid == 0) vecs[0] = mask_vec_outside<kF16>(vecs[0], (int)eoff, 8);
+            if ((end & 7u) != 0 && (last % kCons) == (uint32_t)tid) vecs[last] = mask_vec_outside<kF16>(vecs[last], 0, (int)(end & 7u));
+            if (past < nvec && (past % kCons) == (uint32_t)tid)
+                vecs[past] = make_uint4(El<kF16>::kNegInf2, El<kF16>::kNegInf2, El<kF16>::kNegInf2, El<kF16>::kNegInf2);
+        }
         // where the generated token sits: vector ylocal of this slice (if < nvec), entry yj
-        const uint32_t ylocal = ((uint32_t)ri.y >> 3) - v0;
-        const int yj = ri.y & 7;
+        const uint32_t ylocal = ((eoff + (uint32_t)ri.y) >> 3) - v0;
+        const int yj = (int)((eoff + (uint32_t)ri.y) & 7u);
         const bool label_here = ylocal < nvec;
         const bool owner = label_here && (ylocal % kCons) == (uint32_t)tid;
         const int jy = owner ? (int)(ylocal / kCons) : -1;
@@ -413,6 +499,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
         float Mref = kFloorM;
         if (nvec > 0) {
             uint4 q0 = *(const uint4*)rowbuf;
+            if (kAny) q0 = mask_vec_outside<kF16>(q0, (int)eoff, 8);
             if (label_here && ylocal == 0) q0 = mask_vec_entry<kF16>(q0, yj);
             Mref = max8_scaled<kF16>(q0);
         }
@@ -501,7 +588,7 @@ __global__ void __launch_bounds__(NW * 32 + 32, 1) loss_creg_kernel(CregArgs ca)
         } else {
             // a wait that ran out somewhere in the block ends the block's work here, for all its threads alike
             if (consumer_barrier_or<NW>(aborted)) { aborted = true; break; }
-            tot = dbuf_reduce<NW>(Acc{M, vs, 0.f}, s_part[par], &s_lab[par], warp, lane);
+            tot = creg_reduce<NW>(Acc{M, vs, 0.f}, s_part[par], &s_lab[par], warp, lane);
         }
         float zy_row = s_lab[par].zy;
 

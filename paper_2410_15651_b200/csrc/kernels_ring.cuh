@@ -1,6 +1,7 @@
 // Loss row kernel with a ring of shared-memory chunks, for 16-byte aligned rows outside the range of
-// the two-resident-rows kernel (sm_100a); also the PTX wrappers and per-vector arithmetic that the
-// other row kernels share.
+// the kernel that keeps a row's exponentials on chip (sm_100a): rows shorter than 16 KB, and rows beyond
+// what a cluster of four blocks holds; also the PTX wrappers and per-vector arithmetic that the other row
+// kernels share.
 //
 // Each persistent block owns a ring of 4/8/16 KB slots.  One elected producer thread streams the
 // block's rows into the ring with bulk asynchronous copies (cp.async.bulk, completion counted on an

@@ -56,7 +56,7 @@ def test_lp_new_is_optional(oracle, name, kw):
                                      ("llama2", {"B": 8}),
                                      ("ragged", {"B": 6, "T": 64, "V": 57000}),      # 114 KB rows: cluster of two
                                      ("ragged", {"B": 6, "T": 64, "V": 131072}),     # 256 KB rows: cluster of three
-                                     ("gpt2", {"B": 4, "T": 64}),                    # two-resident-rows kernel
+                                     ("gpt2", {"B": 4, "T": 64}),                    # rows off 16-byte boundaries
                                      ("ragged", {"B": 12, "T": 40, "V": 4096})])     # chunk-ring kernel
 def test_two_runs_are_bit_identical(name, kw):
     # fixed-order reductions, no floating-point atomics: whatever block takes whatever row, and whichever block

@@ -297,8 +297,8 @@ def test_experience_strided_views():
 
 @pytest.mark.parametrize("V,in_place", [(65544, False), (70000, True), (131072, False), (57000, False)])
 def test_rows_larger_than_shared_memory(oracle, V, in_place):
-    # rows above 111 KB are cut into 64 KB tiles and streamed twice: two tiles plus 16 bytes, a ragged last
-    # tile, exactly four tiles; 57000 (114,000 B) is the first size past the two-resident-rows kernel
+    # rows that one block cannot hold twice are shared by a cluster of 2, 3 or 4 blocks: 131,088 B (one vector more
+    # than 128 KB), 140,000 B, exactly 256 KB; 57000 (114,000 B) is the first size that needs a cluster
     w = inputs.scaled(inputs.WORKLOADS["ragged"], V=V, B=5, T=6, seed=70 + V % 7)
     batch = inputs.make_batch(w, device=DEV)
     batch["lengths"] = torch.tensor([0, 1, 6, 3, 6], dtype=torch.int32, device=DEV)
@@ -316,8 +316,8 @@ def test_rows_larger_than_shared_memory(oracle, V, in_place):
 
 @pytest.mark.parametrize("V,in_place", [(32000, False), (50272, True), (4096, False)])
 def test_rows_that_leave_the_common_reference_exponent(oracle, V, in_place):
-    # The loss kernel for rows of 16-111 KB sums a row against one reference exponent taken from the row's first
-    # 8 logits and falls back to per-thread references when that does not hold.  Rows built to force every branch:
+    # The loss kernel sums a row against one reference exponent taken from the row's first 8 logits and falls back to
+    # per-thread references when that does not hold.  Rows built to force every branch:
     # first 8 logits all -inf (no reference); first 8 logits far below the rest (entries > 2^64 above the
     # reference: spikes of +60..+90, at the label and elsewhere); first 8 logits far above the rest (everything else
     # more than 100 binades below the reference); -inf inside the first vector only.  V=4096 takes the chunk-ring kernel.
