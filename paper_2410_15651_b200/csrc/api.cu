@@ -308,7 +308,7 @@ int launch_loss_rows(const RowArgs& a, bool f16, const DeviceInfo& dev, cudaStre
     ra.row_bytes = row_bytes;
     const long long rows = (long long)a.B * a.T;
     const int grid = (int)std::min<long long>(rows, (long long)dev.sm_count * pl.blocks_per_sm);
-    if (pl.NW == 16) return pl.U == 4 ? launch_ring_as<16, 4>(ra, pl, grid, s) : launch_ring_as<16, 2>(ra, pl, grid, s);
+    if (pl.NW == 16) return launch_ring_as<16, 4>(ra, pl, grid, s);
     if (pl.U == 1) return launch_ring_as<8, 1>(ra, pl, grid, s);
     return launch_ring_as<8, 2>(ra, pl, grid, s);
 }

@@ -3,15 +3,14 @@
 // what a cluster of four blocks holds; also the PTX wrappers and per-vector arithmetic that the other row
 // kernels share.
 //
-// Each persistent block owns a ring of 4/8/16 KB slots.  One elected producer thread streams the
+// Each persistent block owns a ring of 4/8/32 KB slots.  One elected producer thread streams the
 // block's rows into the ring with bulk asynchronous copies (cp.async.bulk, completion counted on an
 // mbarrier per slot); NW consumer warps work on the slots as they land and release them through a
 // second mbarrier per slot.
 //
 //   short rows (< 16 KB)     blocks of 8 consumer warps, up to 7 per SM; the row stays in the ring
 //                            ("resident") between the partition-sum pass and the gradient pass.
-//   rows of 111 KB .. 225 KB one block of 16 consumer warps per SM, row resident.
-//   larger rows              streamed twice by one block of 16 consumer warps per SM; the second read
+//   rows beyond a cluster    streamed twice by one block of 16 consumer warps per SM; the second read
 //                            is served by L2.
 //   Padded rows are zero-filled by bulk stores from a zeroed shared buffer, issued by the producer
 //   thread between its loads.
@@ -606,19 +605,7 @@ inline RingPlan plan_ring(unsigned row_bytes, int sm_smem, int block_smem_max)
 {
     constexpr size_t kStatic = 1280;                   // static shared memory of the kernel, rounded up
     constexpr size_t kReserved = 1024;
-    if (row_bytes >= 32768) {
-        // long rows that fit: one block of 16 consumer warps per SM owns all of its shared memory, in
-        // 16 KB chunks; the ring holds the row being processed plus as much of the next as fits, so
-        // loads keep streaming while a row is reduced.
-        const int NW = 16, U = 2;
-        const size_t chunk = (size_t)NW * 32 * 16 * U;
-        const int chunks = (int)((row_bytes + chunk - 1) / chunk);
-        if (ring_smem_bytes(NW, U, chunks) + kStatic <= (size_t)block_smem_max) {
-            int S = chunks;
-            while (ring_smem_bytes(NW, U, S + 1) + kStatic <= (size_t)block_smem_max) ++S;
-            return RingPlan{NW, U, S, chunks, 1, 1, ring_smem_bytes(NW, U, S)};
-        }
-    } else {
+    if (row_bytes < 32768) {
         // short rows: blocks of 8 consumer warps, as many per SM as can hold a row each (at most 7 by
         // thread count); among chunk sizes that reach that count take the preferred one; the ring then
         // grows into what is left.

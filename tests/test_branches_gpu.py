@@ -234,11 +234,13 @@ def test_sequence_shards_reproduce_the_whole_batch(oracle, name, kw, shards):
     assert close_rel(total[0].item(), float(whole.loss[0]))[0]
 
 
-@pytest.mark.parametrize("V", [8192, 8200, 16384, 32768, 32776, 45056, 53248, 57344, 98304, 114688, 163840])
+@pytest.mark.parametrize("V", [8192, 8200, 16384, 32768, 32776, 45056, 53248, 57344, 98304, 114688, 163840,
+                               212992, 213000, 262144])
 def test_vocabulary_sizes_around_the_kernel_boundaries(oracle, V):
     # 16 KB rows (the first size of the on-chip-exponentials kernel), rows that fill a thread's register-held vectors
     # exactly and by one more vector (tensor memory), the last size one block holds twice and the first that needs a
-    # cluster of 2, 3, 4 blocks
+    # cluster of 2, 3, 4 blocks, the last size a cluster of 4 holds, and rows beyond it (425,984 B; 426,000 B and
+    # 512 KB), which the chunk ring streams twice
     from test_parity_gpu import run_steps
     w = inputs.scaled(inputs.WORKLOADS["ragged"], V=V, B=3, T=5, seed=200 + V % 13)
     batch = inputs.make_batch(w, device=DEV)
