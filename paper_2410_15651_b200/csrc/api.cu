@@ -13,6 +13,7 @@
 #include "kernels_generic.cuh"
 #include "kernels_ring.cuh"
 #include "kernels_creg.cuh"
+#include "kernels_cring.cuh"
 #include "kernels_warp.cuh"
 #include "kernels_small.cuh"
 
@@ -262,6 +263,96 @@ int launch_creg_cluster(const RowArgs& a, const CregPlan& pl, const DeviceInfo& 
     }
 }
 
+// The chunk-ring variant of the on-chip-exponentials kernel: a slice may be as long as registers and tensor memory hold
+// exponentials for (8 chunks of 16 KB), so some rows need fewer blocks per cluster than with whole-slice buffers.
+struct CringPlan {
+    int cluster = 0;
+    unsigned slice_vecs = 0, tmem_cols = 0;
+    int n_slots = 0, chunks = 0;
+    size_t smem_bytes = 0;
+};
+
+CringPlan plan_cring(unsigned row_bytes, const DeviceInfo& dev)
+{
+    CringPlan pl;
+    if (row_bytes % 16 != 0) return pl;
+    const unsigned row_vecs = row_bytes / 16;
+    const size_t chunk = cring_chunk_bytes(kCregWarps);
+    int R = kCringMaxSlots;
+    while (R > 0 && cring_smem_bytes(kCregWarps, R) + 3072 > (size_t)dev.max_smem_optin) --R;
+    for (int c = 1; c <= 4; ++c) {
+        const unsigned sv = (row_vecs + c - 1) / c;
+        const int C = (int)(((size_t)sv * 16 + chunk - 1) / chunk);
+        // a slice's chunks stay in the ring from pass 1 to pass 2, and the kernel is fast only while at least five
+        // more slots prefetch the next slice
+        if (C < 3 || C > R - 5 || kCringU * C - kRegVecsTmem > kTmemVecs) continue;
+        if ((size_t)row_vecs <= (size_t)(c - 1) * sv) continue;        // every block of the cluster has a share
+        unsigned cols = 32;
+        while (cols < (unsigned)(kCringU * C - kRegVecsTmem) * 8u * ((kCregWarps + 3) / 4)) cols *= 2;
+        pl.cluster = c;
+        pl.slice_vecs = sv;
+        pl.tmem_cols = cols;
+        pl.n_slots = R;
+        pl.chunks = C;
+        pl.smem_bytes = cring_smem_bytes(kCregWarps, R);
+        return pl;
+    }
+    return pl;
+}
+
+template <int C, bool kF16>
+int launch_cring(const RowArgs& a, const CringPlan& pl, const DeviceInfo& dev, cudaStream_t s)
+{
+    constexpr int NW = kCregWarps;
+    CringArgs ca{};
+    ca.row = a;
+    ca.row_bytes = 2u * (unsigned)a.V;
+    ca.slice_vecs = pl.slice_vecs;
+    ca.tmem_cols = pl.tmem_cols;
+    ca.n_slots = pl.n_slots;
+    ca.chunks = pl.chunks;
+    ca.row_counter = (unsigned*)((char*)a.status + 16);
+    RLHF_CUDA(cudaFuncSetAttribute(loss_cring_kernel<NW, C, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)pl.smem_bytes));
+    // clusters that the device holds at once (one block per SM); looked up once per device
+    static std::mutex mu;
+    static int cached[64] = {};
+    int d = 0, clusters = 0;
+    RLHF_CUDA(cudaGetDevice(&d));
+    if (C == 1) {
+        clusters = dev.sm_count;
+    } else {
+        std::lock_guard<std::mutex> lock(mu);
+        if (d < 0 || d >= 64 || cached[d] == 0) {
+            int n = 0;
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[2];
+            fill_launch_config(cfg, attr, dev.sm_count / C * C, NW * 32 + 32, pl.smem_bytes, C, nullptr);
+            RLHF_CUDA(cudaOccupancyMaxActiveClusters(&n, loss_cring_kernel<NW, C, kF16>, &cfg));
+            if (n < 1) n = 1;
+            if (d >= 0 && d < 64) cached[d] = n;
+            clusters = n;
+        } else {
+            clusters = cached[d];
+        }
+    }
+    const long long rows = (long long)a.B * a.T;
+    const int grid = (int)std::min<long long>(rows, clusters) * C;
+    RLHF_CUDA(launch_kernel_cluster(loss_cring_kernel<NW, C, kF16>, grid, NW * 32 + 32, pl.smem_bytes, C, s, ca));
+    return RLHF_OK;
+}
+
+template <bool kF16>
+int launch_cring_cluster(const RowArgs& a, const CringPlan& pl, const DeviceInfo& dev, cudaStream_t s)
+{
+    switch (pl.cluster) {
+        case 1: return launch_cring<1, kF16>(a, pl, dev, s);
+        case 2: return launch_cring<2, kF16>(a, pl, dev, s);
+        case 3: return launch_cring<3, kF16>(a, pl, dev, s);
+        default: return launch_cring<4, kF16>(a, pl, dev, s);
+    }
+}
+
 // The loss row kernel for 16-byte aligned rows: exponentials kept on chip where the row (or its share in a
 // cluster) fits, else the chunk ring.
 // Rows off 16-byte boundaries: the kernel loads the aligned span around a row, at most 14 bytes before it and 14 after;
@@ -281,17 +372,32 @@ int launch_creg_any(const RowArgs& a, const CregPlan& pl, const DeviceInfo& dev,
                              : launch_creg<kCregWarps, 1, false, kF16, true>(a, pl, dev, s);
 }
 
+// Which of the two takes a row length that both can take.  Measured on V = 57344 ... 256000 (T = 512, 4 GB of logits):
+// the chunk ring wins where it needs fewer blocks per row and at most two (rows of 105-128 KB in one block: 1.02 of the
+// copy rate against 0.86-0.93 in a cluster of two; rows of 210-256 KB in two blocks on all SMs: 0.98 against 0.88-0.92 in
+// three); in clusters of three and four it does not (0.85 against 0.89 at 320 KB), and whole-slice buffers are at their
+// best with slices of 85-105 KB (0.97-1.0).  Rows beyond the largest cluster of whole-slice buffers (426-512 KB) go to
+// the chunk ring in a cluster of four (0.86 against 0.65 for streaming the row twice).
+inline bool use_cring(const CregPlan& cp, const CringPlan& rp)
+{
+    if (rp.cluster == 0) return false;
+    if (cp.cluster == 0) return true;
+    return rp.cluster < cp.cluster && rp.cluster <= 2;
+}
+
 // The fast loss kernels for 16-byte aligned rows of this length (binary16 rows: the on-chip-exponentials kernel
 // only; the chunk ring is a bf16 kernel).
 bool fast_loss_rows_apply(int V, bool f16, const DeviceInfo& dev)
 {
-    return !f16 || plan_creg(2u * (unsigned)V, dev).cluster > 0;
+    return !f16 || plan_cring(2u * (unsigned)V, dev).cluster > 0 || plan_creg(2u * (unsigned)V, dev).cluster > 0;
 }
 
 int launch_loss_rows(const RowArgs& a, bool f16, const DeviceInfo& dev, cudaStream_t s)
 {
     const unsigned row_bytes = 2u * (unsigned)a.V;
     const CregPlan cp = plan_creg(row_bytes, dev);
+    const CringPlan rp = plan_cring(row_bytes, dev);
+    if (use_cring(cp, rp)) return f16 ? launch_cring_cluster<true>(a, rp, dev, s) : launch_cring_cluster<false>(a, rp, dev, s);
     if (cp.cluster > 0) {
         if (f16)
             return cp.tmem_cols != 0 ? launch_creg_cluster<kCregWarps, true, true>(a, cp, dev, s)

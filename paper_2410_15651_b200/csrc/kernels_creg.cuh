@@ -1,6 +1,8 @@
 // Loss forward/backward with the row's exponentials kept on chip between the two passes, for 16-byte
 // aligned rows of 16 KB and more; rows that do not fit one block twice are shared by a thread-block
 // cluster of up to 4 blocks.
+// (kernels_cring.cuh holds the variant that passes the row through a ring of chunks, which takes some row
+// lengths with fewer blocks; the helpers below serve both.)
 //
 // A row's gradient needs every softmax term twice: once in the partition sum and once, scaled by the
 // token's g / sum, as the gradient entry itself.  Recomputing the exponential in the second pass costs two

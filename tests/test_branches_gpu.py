@@ -33,7 +33,8 @@ def _call_loss(w, batch, run, logits, out, ws, grad_scale=None, lengths=None, id
                                      ("llama2", {"B": 2, "T": 24}),                  # exponentials in registers
                                      ("opt", {"B": 2, "T": 24}),                     # registers + tensor memory
                                      ("gpt2", {"B": 2, "T": 12}),                    # rows off 16-byte boundaries
-                                     ("large_vocab", {"B": 1, "T": 12})])            # cluster of three blocks
+                                     ("large_vocab", {"B": 1, "T": 12}),             # two blocks, chunk ring
+                                     ("ragged", {"B": 1, "T": 12, "V": 150000})])    # cluster of three blocks
 def test_lp_new_is_optional(oracle, name, kw):
     w = inputs.scaled(inputs.WORKLOADS[name], **kw)
     batch = inputs.make_batch(w, device=DEV)
@@ -54,8 +55,9 @@ def test_lp_new_is_optional(oracle, name, kw):
 
 @pytest.mark.parametrize("name,kw", [("opt", {}),                                    # rows dealt dynamically, 148 blocks
                                      ("llama2", {"B": 8}),
-                                     ("ragged", {"B": 6, "T": 64, "V": 57000}),      # 114 KB rows: cluster of two
-                                     ("ragged", {"B": 6, "T": 64, "V": 131072}),     # 256 KB rows: cluster of three
+                                     ("ragged", {"B": 6, "T": 64, "V": 57000}),      # 114 KB rows: one block, chunk ring
+                                     ("ragged", {"B": 6, "T": 64, "V": 131072}),     # 256 KB rows: two blocks, chunk ring
+                                     ("ragged", {"B": 6, "T": 64, "V": 150000}),     # 300 KB rows: cluster of three, whole-slice buffers
                                      ("gpt2", {"B": 4, "T": 64}),                    # rows off 16-byte boundaries
                                      ("ragged", {"B": 12, "T": 40, "V": 4096})])     # chunk-ring kernel
 def test_two_runs_are_bit_identical(name, kw):
@@ -234,13 +236,16 @@ def test_sequence_shards_reproduce_the_whole_batch(oracle, name, kw, shards):
     assert close_rel(total[0].item(), float(whole.loss[0]))[0]
 
 
-@pytest.mark.parametrize("V", [8192, 8200, 16384, 32768, 32776, 45056, 53248, 57344, 98304, 114688, 163840,
-                               212992, 213000, 262144])
+@pytest.mark.parametrize("V", [8192, 8200, 16384, 32768, 32776, 45056, 53248, 57344, 65536, 65544, 98304, 106496, 106504, 114688,
+                               131072, 131080, 150000, 163840, 212992, 213000, 262144, 262152])
 def test_vocabulary_sizes_around_the_kernel_boundaries(oracle, V):
     # 16 KB rows (the first size of the on-chip-exponentials kernel), rows that fill a thread's register-held vectors
-    # exactly and by one more vector (tensor memory), the last size one block holds twice and the first that needs a
-    # cluster of 2, 3, 4 blocks, the last size a cluster of 4 holds, and rows beyond it (425,984 B; 426,000 B and
-    # 512 KB), which the chunk ring streams twice
+    # exactly and by one more vector (tensor memory), the last size one block holds twice in whole-row buffers (53248)
+    # and the sizes that one block takes through the chunk ring (57344, 65536: eight full chunks), the first that needs
+    # a cluster of two with whole-slice buffers (65544), the last of those (106496 = 208 KB) and the sizes that two
+    # blocks take through the chunk ring (106504 ... 131072), clusters of three (131080, 150000) and four (163840,
+    # 212992: the last size whole-slice buffers hold), the chunk ring in a cluster of four beyond that (213000, 262144:
+    # 512 KB, eight full chunks per block), and rows beyond everything (262152), which the plain chunk ring streams twice
     from test_parity_gpu import run_steps
     w = inputs.scaled(inputs.WORKLOADS["ragged"], V=V, B=3, T=5, seed=200 + V % 13)
     batch = inputs.make_batch(w, device=DEV)

@@ -34,10 +34,13 @@ def _f16_batch(w):
     ("llama2", {"B": 2, "T": 24}, False),                  # exponentials in registers
     ("opt", {"B": 2, "T": 24}, True),                      # registers + tensor memory, in place
     ("gpt2", {"B": 3, "T": 12, "lengths": "uniform:5:12"}, True),               # rows off 16-byte boundaries
-    ("ragged", {"B": 5, "T": 6, "V": 57000}, False),      # cluster of two blocks
-    ("ragged", {"B": 5, "T": 6, "V": 131072}, False),     # cluster of three blocks
+    ("ragged", {"B": 5, "T": 6, "V": 57000}, False),      # one block, chunk ring
+    ("ragged", {"B": 5, "T": 6, "V": 70000}, False),      # cluster of two blocks, whole-slice buffers
+    ("ragged", {"B": 5, "T": 6, "V": 131072}, False),     # cluster of two blocks, chunk ring
+    ("ragged", {"B": 5, "T": 6, "V": 150000}, False),     # cluster of three blocks
     ("ragged", {"B": 5, "T": 6, "V": 163840}, True),      # cluster of four blocks, in place
-    ("ragged", {"B": 3, "T": 4, "V": 213000}, False),     # beyond a cluster: generic kernel for fp16
+    ("ragged", {"B": 3, "T": 4, "V": 213000}, False),     # cluster of four blocks, chunk ring
+    ("ragged", {"B": 3, "T": 4, "V": 262152}, False),     # beyond every cluster: generic kernel for fp16
     ("ragged", {"B": 12, "T": 40, "V": 16384}, False),    # -inf entries, sharpened rows, 32 KB rows
 ])
 def test_fp16_logits_every_step(oracle, name, kw, in_place):

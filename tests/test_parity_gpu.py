@@ -297,8 +297,8 @@ def test_experience_strided_views():
 
 @pytest.mark.parametrize("V,in_place", [(65544, False), (70000, True), (131072, False), (57000, False)])
 def test_rows_larger_than_shared_memory(oracle, V, in_place):
-    # rows that one block cannot hold twice are shared by a cluster of 2, 3 or 4 blocks: 131,088 B (one vector more
-    # than 128 KB), 140,000 B, exactly 256 KB; 57000 (114,000 B) is the first size that needs a cluster
+    # rows that one block cannot hold twice in whole-row buffers: 131,088 B (one vector more than 128 KB) and 140,000 B
+    # go to a cluster of two, exactly 256 KB to two blocks with a chunk ring each, 114,000 B to one such block
     w = inputs.scaled(inputs.WORKLOADS["ragged"], V=V, B=5, T=6, seed=70 + V % 7)
     batch = inputs.make_batch(w, device=DEV)
     batch["lengths"] = torch.tensor([0, 1, 6, 3, 6], dtype=torch.int32, device=DEV)
