@@ -45,11 +45,11 @@ AUX_STEPS = {"llama2": 1000, "large_vocab": 100, "ragged": 120, "gpt2": 1500, "o
 
 # DRAM traffic per launch of the loss kernel (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed
 # by workload; reported only while the kernel sources still hash to the value the captures were taken at, else null.
-# The summaries and their commands are profiles/loss_creg_kernel_opt.md and profiles/loss_creg_kernel_large_vocab_8seq.md;
-# the large-vocabulary figure is the 8-sequence capture (1050.886 MB + 998.257 MB) times 8, the bench's workload having
+# The summaries and their commands are profiles/loss_creg_kernel_opt.md and profiles/loss_cring_kernel_large_vocab_8seq.md;
+# the large-vocabulary figure is the 8-sequence capture (1050.897 MB + 996.266 MB) times 8, the bench's workload having
 # 8 times the rows (rows are independent and streamed once each, so traffic grows in proportion).
-NCU_TRAFFIC = {"sources_sha256": "852593ca1b344c8c",
-               "bytes_per_launch": {"opt": 302417920 + 356522240, "large_vocab": 8 * (1050886000 + 998256640)}}
+NCU_TRAFFIC = {"sources_sha256": "1b545b70514a9280",
+               "bytes_per_launch": {"opt": 302417920 + 357586944, "large_vocab": 8 * (1050897000 + 996265984)}}
 
 
 def sources_digest() -> str:
