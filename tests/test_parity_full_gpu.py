@@ -6,9 +6,11 @@ Every O(B*T) output (log-probs of all rows for actor and reference, rewards, adv
 dvalues, both losses) is compared in full: the oracle computes all of them.  The bf16 logits
 gradient is compared element by element on every row for the OPT- and Llama-2-shaped workloads
 (out of place), and for the others on a sample of rows (valid, padded, zero-gradient, first and
-last, and for the large-vocabulary workload, whose rows are dealt statically to clusters of blocks,
-the first and the last 64 valid rows, which covers every cluster at the start and at the end of
-its work); every row is also checked through properties that need no oracle row.
+last, and for the large-vocabulary workload, whose rows are dealt statically to 74 clusters of two
+blocks with a ring of 13 chunk slots each (a slice takes 8, so a cluster's i-th row starts at slot
+8i mod 13), the first 1024 valid rows, which cover every block at every ring offset and both
+phases of every slot's barriers, and the last 148, the end of every cluster's work); every row is
+also checked through properties that need no oracle row.
 """
 import numpy as np
 import pytest
@@ -31,7 +33,7 @@ def test_full_size(oracle, name, in_place):
     rows = sample_rows(run, 48, seed=w.seed)
     if name == "large_vocab":
         flat_valid = np.flatnonzero(run.valid.reshape(-1))
-        rows = np.unique(np.concatenate([rows, flat_valid[:64], flat_valid[-64:]]))
+        rows = np.unique(np.concatenate([rows, flat_valid[:1024], flat_valid[-148:]]))
     every_row = name in ("opt", "llama2") and not in_place
     out, rep = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"],
                          in_place=in_place, sample_rows=rows, all_rows=every_row)
