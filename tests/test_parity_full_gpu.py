@@ -4,9 +4,9 @@ configuration the benchmark times.
 
 Every O(B*T) output (log-probs of all rows for actor and reference, rewards, advantages, returns,
 dvalues, both losses) is compared in full: the oracle computes all of them.  The bf16 logits
-gradient is compared element by element on every row for the OPT- and Llama-2-shaped workloads
-(out of place), and for the others on a sample of rows (valid, padded, zero-gradient, first and
-last, and for the large-vocabulary workload, whose rows are dealt statically to 74 clusters of two
+gradient is compared element by element on every row for the OPT-, Llama-2- and GPT-2-shaped workloads
+(out of place), and for the others on a sample of rows (some 600 for the ragged workload; valid,
+padded, zero-gradient, first and last, and for the large-vocabulary workload, whose rows are dealt statically to 74 clusters of two
 blocks with a ring of 13 chunk slots each (a slice takes 8, so a cluster's i-th row starts at slot
 8i mod 13), the first 1024 valid rows, which cover every block at every ring offset and both
 phases of every slot's barriers, and the last 148, the end of every cluster's work); every row is
@@ -34,7 +34,9 @@ def test_full_size(oracle, name, in_place):
     if name == "large_vocab":
         flat_valid = np.flatnonzero(run.valid.reshape(-1))
         rows = np.unique(np.concatenate([rows, flat_valid[:1024], flat_valid[-148:]]))
-    every_row = name in ("opt", "llama2") and not in_place
+    if name == "ragged":
+        rows = np.unique(np.concatenate([rows, sample_rows(run, 600, seed=w.seed + 1)]))
+    every_row = name in ("opt", "llama2", "gpt2") and not in_place
     out, rep = run_steps(oracle, w, batch, run, batch["actor"], batch["ref"], batch["ids"],
                          in_place=in_place, sample_rows=rows, all_rows=every_row)
     dlogits_properties(run, out, batch["ids"], batch["actor"])
